@@ -209,7 +209,10 @@ rpa_status_t rpa_forward_host_wait(rpa_handle_t* h);
  * a device share the one array, which keeps the previous call's contents (nothing in it needs
  * clearing: a call reads only what it wrote itself).  Host-side, calls are serialised by a lock;
  * on the GPU, two calls that overlap in time (different streams) race on the array -- keep calls
- * on one device ordered on a single stream.
+ * on one device ordered on a single stream.  The work lists of a call are copied from ordinary host
+ * memory, so the call returns only after earlier work on `stream` has finished (the kernels it
+ * enqueues run asynchronously as usual); a stream that is being captured is refused with
+ * RPA_ERR_UNSUPPORTED, as are head_dim 256 and an FP8 cache.
  */
 rpa_status_t rpa_forward_static(const rpa_config_t* cfg, const void* q, const void* new_k, const void* new_v,
                                 void* kv_cache, const int32_t* page_table, const int32_t* cu_q_lens,

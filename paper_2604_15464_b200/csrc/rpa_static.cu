@@ -75,6 +75,16 @@ extern "C" rpa_status_t rpa_forward_static(const rpa_config_t* cfg, const void* 
         cfg->kv_dtype != RPA_KV_BF16)
         return RPA_ERR_UNSUPPORTED;
 
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    // The work lists travel from ordinary (pageable) host memory.  On a stream that executes, the
+    // runtime has read the bytes by the time the copy call returns, so g_plan may be reused at once;
+    // the price is that the call waits for earlier work on `stream`.  A stream that is being captured
+    // would instead record g_plan's address in the graph and read it at every replay, long after the
+    // plan has changed: such a stream is refused.
+    cudaStreamCaptureStatus capture = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(s, &capture) != cudaSuccess) return RPA_ERR_CUDA;
+    if (capture != cudaStreamCaptureStatusNone) return RPA_ERR_UNSUPPORTED;
+
     std::lock_guard<std::mutex> lock(g_mutex);
     int dev = -1;
     cudaError_t e = cudaGetDevice(&dev);
@@ -105,8 +115,6 @@ extern "C" rpa_status_t rpa_forward_static(const rpa_config_t* cfg, const void* 
         return RPA_ERR_INVALID_ARG;
 
     unsigned char* scratch = g_scratch_ptr[dev];
-    cudaStream_t s = static_cast<cudaStream_t>(stream);
-    // pageable source: the runtime stages the bytes before returning, so g_plan may be reused at once
     e = cudaMemcpyAsync(scratch + kOffRows, g_plan.rows.data(), g_plan.rows.size() * sizeof(RowItem),
                         cudaMemcpyHostToDevice, s);
     if (e == cudaSuccess && !g_plan.groups.empty())

@@ -172,7 +172,7 @@ rpa_tile1_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
                 if (q_prefetched_for != iter)  // the CTA's first item (later ones were loaded during their predecessor)
                     load_q(smem_base + q_off, bar(T1_Q + (iter & 1)), h, cu + it.q_tok0);
             }
-            const int box_rows = min(ps, BN);
+            const int box_rows = page_box_rows(ps, BN);
             const int sub_blocks = BN / box_rows;
             bool ok = true;
             for (int j = 0; j < n_blocks && ok; ++j) {
@@ -337,7 +337,7 @@ rpa_tile1_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
                 // stage) into the 64-column blocks of the bf16 operand layout, every E4M3 value
                 // being exact in bf16.  Blocks 2b and 2b+1 come from raw row b; the last ones land
                 // on raw rows this thread has read by then.
-                const int t = tid - 64, box_rows = min(ps, BN);
+                const int t = tid - 64, box_rows = page_box_rows(ps, BN);
                 bool okc = true;
                 for (int j = 0; j < n_ctx_blocks && okc; ++j) {
                     const int st = j & 1, ph = (j >> 1) & 1;

@@ -15,8 +15,17 @@ struct TileMaps {
     CUtensorMap out;    // same geometry as q
     CUtensorMap new_k;  // (d, h_kv, T)    box (64, 1, key-block positions)
     CUtensorMap new_v;
-    CUtensorMap cache;  // (d, 2h_kv, page_size, num_pages)  box (64, 1, min(page_size, key-block positions), 1)
+    CUtensorMap cache;  // (d, 2h_kv, page_size, num_pages)  box (64, 1, page_box_rows(page_size, key-block positions), 1)
 };
+
+// Rows of one per-page TMA box of a context key block.  A block of block_n positions is fetched as
+// block_n / rows boxes, each starting at a position that is a multiple of `rows`; `rows` divides
+// both the page size and the block, so no box straddles a page whatever the page size is (48, 96,
+// 192, ... included): the largest power of two that divides page_size, capped at the block.
+__host__ __device__ __forceinline__ int page_box_rows(int page_size, int block_n) {
+    const int pow2 = page_size & -page_size;
+    return pow2 < block_n ? pow2 : block_n;
+}
 
 // Everything a role needs to know about one work item.
 struct TileCtx {
@@ -279,12 +288,12 @@ inline bool build_tile_maps(const KernelArgs& a, int64_t token_rows, int D, int 
         // one-byte elements: 128 codes are one 128-byte swizzle span (a row of d_k = 256 takes two boxes)
         const uint64_t dims[4] = {d, (uint64_t)2 * a.h_kv, (uint64_t)a.page_size, (uint64_t)a.num_pages};
         const uint64_t str[3] = {d, d * 2 * a.h_kv, d * 2 * a.h_kv * a.page_size};
-        const uint32_t box[4] = {128, 1, (uint32_t)(a.page_size < block_n ? a.page_size : block_n), 1};
+        const uint32_t box[4] = {128, 1, (uint32_t)page_box_rows(a.page_size, block_n), 1};
         if (D % 128 || !make_map(&maps->cache, a.kv_cache, 4, dims, str, box, CU_TENSOR_MAP_DATA_TYPE_UINT8)) return false;
     } else {
         const uint64_t dims[4] = {d, (uint64_t)2 * a.h_kv, (uint64_t)a.page_size, (uint64_t)a.num_pages};
         const uint64_t str[3] = {d * 2, d * 2 * 2 * a.h_kv, d * 2 * 2 * a.h_kv * a.page_size};
-        const uint32_t box[4] = {64, 1, (uint32_t)(a.page_size < block_n ? a.page_size : block_n), 1};
+        const uint32_t box[4] = {64, 1, (uint32_t)page_box_rows(a.page_size, block_n), 1};
         if (!make_map(&maps->cache, a.kv_cache, 4, dims, str, box)) return false;
     }
     return true;

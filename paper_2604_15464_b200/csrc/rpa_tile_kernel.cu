@@ -190,7 +190,7 @@ rpa_tile_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
             if (q_prefetched_for != iter)  // the CTA's first item (later ones were loaded during their predecessor)
                 load_q(q_region, bar(BAR_Q + (iter & 1)), it.n_tok, h, cu + it.q_tok0);
         }
-        const int box_rows = min(ps, kBlockN);
+        const int box_rows = page_box_rows(ps, kBlockN);
         const int sub_blocks = kBlockN / box_rows;
         bool ok = true;
         for (int j = 0; j < n_blocks && ok; ++j) {
@@ -480,7 +480,7 @@ rpa_tile_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
             // the bf16 operand layout, every E4M3 value being exact in bf16.  The second half lands
             // on the raw row itself, which the thread has read by then.
             static_assert(!FP8 || D == 128, "raw rows of 128 bytes");
-            const int t = tid - 64, box_rows = min(ps, kBlockN);
+            const int t = tid - 64, box_rows = page_box_rows(ps, kBlockN);
             bool okc = true;
             for (int j = 0; j < n_ctx_blocks && okc; ++j) {
                 const int st = j & 1, ph = (j >> 1) & 1;

@@ -12,6 +12,8 @@ bf16, synthetic batches) with raggedness added:
   3  full causal prefill, 4 requests of 8192 tokens, page 128
   4  mixed: 192 decode requests (kv_len ~ U{256..8192}) + 8 chunks of 512 new tokens on a prior
      context ~ U{0..4096}, page 16, token capacity 8192
+  "4b"  the same with chunks of 1000 tokens: 192 + 8000 = 8192 new tokens, exactly the capacity, and
+     chunk lengths that are no multiple of a query tile
   5  skewed decode: 512 requests, log-normal kv_len (median 2048, sigma 1.5, cap 131072), page 128,
      pages scattered over a pool sized by the caller
 """
@@ -125,9 +127,13 @@ def build_meta(name: str, q_lens: Sequence[int], kv_lens: Sequence[int], *, num_
 LLAMA3_8B = dict(num_q_heads=32, num_kv_heads=8, head_dim=128)
 
 
-def workload_meta(config: int, seed: Optional[int] = None, *, num_pages: Optional[int] = None,
+def workload_meta(config, seed: Optional[int] = None, *, num_pages: Optional[int] = None,
                   sigma: float = 1.5) -> BatchMeta:
-    """Metadata of named workload ``config`` (1..5).  ``seed`` defaults to 1000 + config."""
+    """Metadata of named workload ``config`` (1..5, or "4b").  ``seed`` defaults to 1000 + config
+    (1004 for "4b": the same decode requests and contexts as workload 4)."""
+    chunk = 512
+    if config == "4b":
+        config, chunk = 4, 1000
     seed = 1000 + config if seed is None else seed
     rng = np.random.default_rng(seed)
     if config == 1:
@@ -143,10 +149,11 @@ def workload_meta(config: int, seed: Optional[int] = None, *, num_pages: Optiona
     if config == 4:
         dec_kv = rng.integers(256, 8192, size=192, endpoint=True)
         ctx = rng.integers(0, 4096, size=8, endpoint=True)
-        q = np.concatenate([np.ones(192, dtype=np.int64), np.full(8, 512)])
-        kv = np.concatenate([dec_kv, ctx + 512])
+        q = np.concatenate([np.ones(192, dtype=np.int64), np.full(8, chunk)])
+        kv = np.concatenate([dec_kv, ctx + chunk])
         order = rng.permutation(200)  # requests arrive interleaved; nothing downstream may rely on an order
-        return build_meta("llama3_8b_mixed", q[order], kv[order], page_size=16, seed=seed, token_capacity=8192,
+        name = "llama3_8b_mixed" if chunk == 512 else f"llama3_8b_mixed_chunk{chunk}"
+        return build_meta(name, q[order], kv[order], page_size=16, seed=seed, token_capacity=8192,
                           num_pages=num_pages, **LLAMA3_8B)
     if config == 5:
         kv = np.exp(math.log(2048.0) + sigma * rng.standard_normal(512))

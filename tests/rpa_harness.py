@@ -86,13 +86,24 @@ def host_subset(batch, seqs):
     return host, oracle_shape(batch.meta, num_pages=n_pages), rows, pages
 
 
-def sampled_parity(batch, seqs, rows_per_seq=None, *, rng=None, rapi=None, kv_chunk=0, tile_min_q=None):
+def sampled_parity(batch, seqs, rows_per_seq=None, *, rng=None, rapi=None, kv_chunk=0, tile_min_q=None,
+                   whole_cache=False):
     """Run the full batch on the GPU, check the sampled sequences' outputs and cache pages against
-    the oracle (all their rows, or ``rows_per_seq`` random (token, head) pairs each)."""
+    the oracle (all their rows, or ``rows_per_seq`` random (token, head) pairs each).  With
+    ``whole_cache`` every byte of the pool is compared as well: the oracle's update step (a bit copy
+    per new token) is applied to a host copy of the whole cache taken before the call, so slots the
+    call must leave alone are covered too."""
     meta = batch.meta
     rng = rng or np.random.default_rng(0)
     host, shape, rows, pages = host_subset(batch, seqs)  # snapshot BEFORE the call
+    whole = None
+    if whole_cache:
+        whole = wl.bf16_bits(batch.kv_cache).copy()
+        orc.update_cache(oracle_shape(meta), wl.bf16_bits(batch.new_k), wl.bf16_bits(batch.new_v), whole, meta.page_table,
+                         meta.cu_q_lens, meta.kv_lens)
     got, info = run_gpu(batch, kv_chunk=kv_chunk, rapi=rapi, tile_min_q=tile_min_q)
+    if whole is not None:
+        assert np.array_equal(wl.bf16_bits(batch.kv_cache), whole), "the pool differs from the oracle's somewhere"
     orc.update_cache(shape, host["new_k"], host["new_v"], host["kv_cache"], host["page_table"], host["cu_q_lens"],
                      host["kv_lens"])
     idx = torch.tensor(pages, dtype=torch.long, device=batch.kv_cache.device)

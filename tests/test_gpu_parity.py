@@ -168,27 +168,62 @@ def test_llama_decode_full_batch():
 
 def test_llama_prefill_sampled_rows():
     batch = wl.materialize(wl.workload_meta(3), _dev())
-    (mx, mean), info = hz.sampled_parity(batch, seqs=[0, 3], rows_per_seq=192)
+    (mx, mean), info = hz.sampled_parity(batch, seqs=[0, 3], rows_per_seq=192, whole_cache=True)
     assert info["batch_case_name"] == "prefill"
+
+
+def _mixed_sample(meta):
+    prefill = [r for r in range(meta.num_seqs) if meta.q_lens[r] > 1]
+    decode = [r for r in range(meta.num_seqs) if meta.q_lens[r] == 1]
+    return prefill[:3] + decode[:12]
 
 
 def test_llama_mixed_sampled_rows():
     meta = wl.workload_meta(4)
     batch = wl.materialize(meta, _dev())
-    prefill = [r for r in range(meta.num_seqs) if meta.q_lens[r] > 1]
-    decode = [r for r in range(meta.num_seqs) if meta.q_lens[r] == 1]
-    seqs = prefill[:3] + decode[:12]
-    (mx, mean), info = hz.sampled_parity(batch, seqs=seqs, rows_per_seq=128)
+    (mx, mean), info = hz.sampled_parity(batch, seqs=_mixed_sample(meta), rows_per_seq=128, whole_cache=True)
     assert info["batch_case_name"] == "mixed" and info["num_tokens"] == 4288
 
 
-def test_skewed_long_decode_sampled_requests():
-    meta = wl.workload_meta(5)
+def test_llama_mixed_1000_token_chunks_fill_the_token_capacity():
+    # 192 decode requests + 8 chunks of 1000 tokens = 8192 new tokens = the capacity of q / new_k / new_v / out;
+    # 1000 is no multiple of a query tile (32 tokens) nor of an item (64)
+    meta = wl.workload_meta("4b")
+    assert meta.num_tokens == 8192 == meta.token_capacity
+    batch = wl.materialize(meta, _dev())
+    (mx, mean), info = hz.sampled_parity(batch, seqs=_mixed_sample(meta), rows_per_seq=160, whole_cache=True)
+    assert info["batch_case_name"] == "mixed" and info["num_tokens"] == 8192
+
+
+def _bench_pool_pages():
+    """The pool bench.py gives the skewed workload: min(150 GB, 0.8 x free HBM) of 512-KB pages."""
+    torch.cuda.empty_cache()
+    free, _ = torch.cuda.mem_get_info()
+    return int(min(150e9, 0.8 * free) // (128 * 2 * 8 * 128 * 2))
+
+
+@pytest.mark.parametrize("sigma", [1.5, 2.0])
+def test_skewed_long_decode_sampled_requests(sigma):
+    # the timed configuration: mapped pages drawn from the whole ~150 GB pool (only they hold random
+    # values; the rest of the pool is a constant)
+    meta = wl.workload_meta(5, num_pages=_bench_pool_pages(), sigma=sigma)
+    assert meta.page_table.max() > 0.9 * meta.num_pages  # ids reach the far end of the pool
     batch = wl.materialize(meta, _dev())
     order = np.argsort(meta.kv_lens)
     seqs = [int(order[-1]), int(order[-2]), int(order[0]), int(order[len(order) // 2]), int(order[len(order) // 3])]
     (mx, mean), info = hz.sampled_parity(batch, seqs=seqs)
     assert info["num_combine_groups"] > 0  # the longest requests were split
+    # slots the call must leave alone: every page of the pool that no request maps still holds the
+    # fill constant (the sampled requests' pages were compared with the oracle's, bit for bit, above)
+    mapped = torch.zeros(meta.num_pages, dtype=torch.bool, device=_dev())
+    mapped[torch.from_numpy(meta.mapped_pages().astype(np.int64)).to(_dev())] = True
+    raw = batch.kv_cache.view(torch.int16)
+    step = 2048  # pages per pass (1 GB)
+    for p0 in range(0, meta.num_pages, step):
+        dirty = (raw[p0:p0 + step] != 0x3F00).flatten(1).any(1)
+        assert not bool((dirty & ~mapped[p0:p0 + step]).any()), f"an unmapped page near {p0} was written"
+    del batch
+    torch.cuda.empty_cache()
 
 
 # ---- edge cases ----

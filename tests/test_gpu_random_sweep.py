@@ -86,3 +86,19 @@ def test_random_batches_with_short_prompts_and_device_planning(seed):
                          kv_fp8=fp8, k_scale=0.03 if fp8 else 1.0, v_scale=0.025 if fp8 else 1.0, **case)
     batch = wl.materialize(meta, torch.device("cuda", 0), canaries=bool(rng.integers(0, 3) == 0))
     hz.full_parity(batch, device_plan=device_plan)
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_random_batches_on_unaligned_page_sizes(seed):
+    """The same draw on page sizes that are multiples of 16 but neither divide nor are a multiple of
+    a key block of the tile kernels (64 or 128 positions)."""
+    rng = np.random.default_rng(5000 + seed)
+    case = _random_case(rng, n_max=9, kinds=5)
+    case["page_size"] = int(rng.choice([48, 80, 96, 112, 144, 176, 192, 240]))
+    q_lens, kv_lens = case.pop("q_lens"), case.pop("kv_lens")
+    fp8 = bool(rng.integers(0, 3) == 0)
+    meta = wl.build_meta(f"randu{seed}", q_lens, kv_lens, seed=500 + seed, token_capacity=sum(q_lens) + 3,
+                         kv_fp8=fp8, k_scale=0.03 if fp8 else 1.0, v_scale=0.025 if fp8 else 1.0, **case)
+    tile_min_q = [None, 1, 8][seed % 3]
+    batch = wl.materialize(meta, torch.device("cuda", 0), canaries=bool(seed % 2))
+    hz.full_parity(batch, tile_min_q=tile_min_q, device_plan=(tile_min_q is None and seed % 4 == 0))

@@ -139,3 +139,19 @@ def test_mixed_routing_uses_both_kernels():
                          page_size=16, seed=16)
     _, info = hz.full_parity(wl.materialize(meta, _dev()))
     assert info["num_tile_items"] > 0 and info["num_row_items"] > 0
+
+
+# Page sizes that neither divide a key block nor are a multiple of one (48, 80, 96, 112, 144, 192):
+# a key block then spans pages at offsets that are not block-aligned, and the per-page boxes of the
+# context gather must follow the page boundaries, not the block's.
+@pytest.mark.parametrize("ps", [48, 80, 96, 112, 144, 192])
+@pytest.mark.parametrize("d,fp8", [(128, False), (128, True), (256, False), (256, True), (64, False)])
+def test_tile_kernels_on_page_sizes_that_do_not_align_with_key_blocks(ps, d, fp8):
+    extra = dict(kv_fp8=True, k_scale=0.03, v_scale=0.025) if fp8 else {}
+    h_q, h_kv = (32, 8) if d != 64 else (8, 2)
+    meta = wl.build_meta(f"ps{ps}", [70, 16, 40, 1], [70 + 5 * ps + 7, 16 + 1000, 40 + ps, 2 * ps + 1], num_q_heads=h_q,
+                         num_kv_heads=h_kv, head_dim=d, page_size=ps, seed=23 + ps, **extra)
+    _, info = hz.full_parity(wl.materialize(meta, _dev(), canaries=True), tile_min_q=1)
+    assert info["num_tile_items"] > 0
+    # and with the default routing (row kernel for the decode row)
+    hz.full_parity(wl.materialize(meta, _dev()))
