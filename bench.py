@@ -7,7 +7,18 @@ decode batch (256 requests, kv_len ~ U{512..4096}, page 16); its metric is the a
 throughput in GB/s on the algorithmic bytes of the paper's decode-throughput formula (Section
 4.1.1) generalised to ragged batches.  Other workloads: ``--workload prefill|mixed|skewed``.
 
+By default one invocation times all three legs of the metric: the decode batch is the headline line
+and the Llama-3-8B-shaped prefill (4 x 8192 tokens, TFLOP/s) and mixed (192 decode + 8 x 512-token
+chunks, tokens/s) batches ride along under ``"legs"``, each with its own value, roofline, end-to-end
+figure, CPU baseline and clock samples.  ``--workload NAME`` runs one workload only.
+
+Timing: W warm-up steps, then blocks of exactly K steps, each bracketed by CUDA events (and, under
+torchrun, a barrier); blocks are repeated until at least ``--min-seconds`` of GPU time has been timed,
+and the median block is reported.  Clock samples are taken while those blocks run.  Per-kernel event
+pairs are off during the timed blocks; the kernel durations of the roofline come from a second pass.
+
 One JSON line is printed (rank 0).  ``--impl reference`` times the fp64 CPU oracle instead.
+``--gpus N`` without a torchrun environment re-executes itself under ``torch.distributed.run``.
 """
 from __future__ import annotations
 
@@ -34,6 +45,7 @@ WORKLOADS = {
     "decode": (2, "decode_hbm_throughput", "GB/s", "hbm"),
     "prefill": (3, "prefill_tensor_throughput", "TFLOP/s", "tensor"),
     "mixed": (4, "mixed_batch_tokens_per_s", "tokens/s", "hbm"),
+    "mixed4b": ("4b", "mixed_batch_tokens_per_s", "tokens/s", "hbm"),  # chunks of 1000 tokens: 8192 new tokens
     "skewed": (5, "decode_hbm_throughput", "GB/s", "hbm"),
     # the paper's own uniform grids (Section 4.1.1 and 4.2.1: page 256, Llama-3-8B heads), --ctx / --seq
     "paper_decode": (0, "decode_hbm_throughput", "GB/s", "hbm"),
@@ -132,7 +144,7 @@ def make_meta(workload: str, rank: int, pool_gb: float | None, args=None):
     by_heads = args is not None and getattr(args, "shard", "requests") == "heads"
     # sharding by request: every rank draws its own batch of the same shape (weak scaling);
     # sharding by KV head: all ranks see the same requests and split the heads (strong scaling)
-    seed = 1000 + cfg + (0 if by_heads else 7919 * rank)
+    seed = 1000 + (4 if cfg == "4b" else cfg) + (0 if by_heads else 7919 * rank)
     if workload == "paper_decode":  # n = 128 requests of identical context length, one new token each
         n, ctx = args.paper_n or 128, args.ctx
         shape = dict(wl.LLAMA3_8B, head_dim=args.head_dim)
@@ -264,62 +276,52 @@ def device_plan_launches(meta):
     return 1 + rows + tiles
 
 
-def main():
-    ap = argparse.ArgumentParser()
-    ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
-    ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="decode", choices=sorted(WORKLOADS))
-    ap.add_argument("--pool-gb", type=float, default=None, help="cache pool size for the skewed workload")
-    ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--no-e2e", action="store_true")
-    ap.add_argument("--kv-chunk", type=int, default=0)
-    ap.add_argument("--ablate", type=int, default=0, help="rpa_set_ablation mask (1: no cache update, 2: no kernel overlap, 4: no attention arithmetic, 8: no K/V loads)")
-    ap.add_argument("--ctx", type=int, default=8192, help="context length of the paper_decode workload")
-    ap.add_argument("--seq", type=int, default=8192, help="sequence length of the paper_prefill workload")
-    ap.add_argument("--paper-n", type=int, default=0, help="requests in the paper_* workloads (default 128 / 1)")
-    ap.add_argument("--page-size", type=int, default=256, help="page size of the paper_* workloads")
-    ap.add_argument("--noncausal", action="store_true", help="paper_* workloads without the causal mask")
-    ap.add_argument("--head-dim", type=int, default=128, help="head dimension of the paper_* workloads (128 or 256)")
-    ap.add_argument("--kv-fp8", action="store_true", help="FP8 E4M3 cache with per-tensor scales (decode workloads)")
-    ap.add_argument("--plan", default="host", choices=["host", "device"],
-                    help="who builds the work lists each step: rpa_plan on the host, or rpa_plan_device on the GPU")
-    ap.add_argument("--shard", default="requests", choices=["requests", "heads"],
-                    help="how N ranks split the work: own requests each (weak scaling) or own KV heads each (strong)")
-    args = ap.parse_args()
-    args.warmup = max(args.warmup, 3)
+def median(xs):
+    xs = sorted(xs)
+    return xs[len(xs) // 2] if len(xs) % 2 else 0.5 * (xs[len(xs) // 2 - 1] + xs[len(xs) // 2])
 
-    if args.impl == "reference":
-        return run_reference(args)
 
-    from paper_2604_15464_b200 import binding, build
+def timed_blocks(run_block, steps, min_seconds, dist, device, max_blocks=4000):
+    """Runs blocks of exactly ``steps`` steps until ``min_seconds`` of GPU time has been timed (at
+    least one block, at most ``max_blocks``).  Every block is bracketed by a synchronize (and a barrier
+    under torchrun) on both sides and timed with CUDA events on the launching stream; a block's time is
+    the slowest rank's.  Returns the per-block times in ms."""
+    stream = torch.cuda.current_stream()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    times, total = [], 0.0
+    while len(times) < max_blocks:
+        if dist:
+            dist.barrier()
+        torch.cuda.synchronize()
+        e0.record(stream)
+        run_block(steps)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1)
+        if dist:  # all ranks must agree on the block's time, hence on when to stop
+            t = torch.tensor([ms], device=device, dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        times.append(ms)
+        total += ms
+        if total >= 1e3 * min_seconds:
+            break
+    return times
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    if not torch.cuda.is_available():
-        raise RuntimeError("bench.py needs a CUDA device: the product has no CPU path")
-    torch.cuda.set_device(local)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
 
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-    if rank == 0:
-        build.build()
-    if dist:
-        dist.barrier()
-    binding.load_library()
+def run_leg(workload, args, rank, world, local, dist, peaks):
+    """Everything bench.py reports for one workload; returns the dict of its JSON line (rank 0's view)."""
+    from paper_2604_15464_b200 import binding
 
-    cfg, metric, unit, bound = WORKLOADS[args.workload]
-    meta = make_meta(args.workload, rank, args.pool_gb, args)
+    device = torch.device("cuda", local)
+    cfg, metric, unit, bound = WORKLOADS[workload]
+    meta = make_meta(workload, rank, args.pool_gb, args)
     if args.shard == "heads" and world > 1:
         meta = shard_heads(meta, rank, world)
     if args.kv_fp8:
         meta.kv_fp8, meta.k_scale, meta.v_scale = True, 0.02, 0.02
         meta.name += "_fp8kv"
-    batch = wl.materialize(meta, torch.device("cuda", local))
+    batch = wl.materialize(meta, device)
     rapi = binding.Rpa.for_meta(meta, device=local)
     if args.kv_chunk:
         rapi.rpa_set_kv_chunk(args.kv_chunk)
@@ -348,39 +350,30 @@ def main():
             rapi.rpa_plan_device(batch.cu_q_lens, batch.kv_lens, plan_stream.cuda_stream)
             planned_ahead[0] = True
 
+    def run_steps(k):
+        for _ in range(k):
+            step()
+
     rapi.rpa_plan(cu_h, kl_h, sh)  # the counts reported below come from the host planner in either mode
     info = rapi.rpa_plan_info()
     planned_ahead[0] = False
-    for _ in range(args.warmup):
-        step()
+    run_steps(args.warmup)
     torch.cuda.synchronize()
 
-    # ---- timed region: device-resident inputs ----
-    if dist:
-        dist.barrier()
-    torch.cuda.synchronize()
-    rapi.rpa_set_kernel_timing(True)
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    # ---- timed region: device-resident inputs, per-kernel events off, clocks sampled while it runs ----
     with ClockSampler(physical_gpu_index(local)) as clocks:
-        e0.record(stream)
-        for _ in range(args.steps):
-            step()
-        e1.record(stream)
-        torch.cuda.synchronize()
-        kt = rapi.rpa_get_kernel_timing()
-        rapi.rpa_set_kernel_timing(False)
-        if e0.elapsed_time(e1) < 600.0:  # keep the GPU under the same load until a few clock samples exist
-            t_end = time.time() + 0.7
-            while time.time() < t_end:
-                step()
-            torch.cuda.synchronize()
-    ms_total, units_per_step = aggregate_over_ranks(e0.elapsed_time(e1), units_of(args.workload, info, meta), dist,
-                                                    torch.device("cuda", local))
-    ms_per_step = ms_total / args.steps
+        block_ms = timed_blocks(run_steps, args.steps, args.min_seconds, dist, device)
+    _, units_per_step = aggregate_over_ranks(0.0, units_of(workload, info, meta), dist, device)
+    ms_per_step = median(block_ms) / args.steps
     value = units_per_step / (ms_per_step * 1e-3)
 
-    # ---- roofline of the dominant kernel (this rank), timed live with events around its launches ----
-    peaks = load_peaks()
+    # ---- roofline of the dominant kernel (this rank): a second pass with event pairs around each launch ----
+    rapi.rpa_set_kernel_timing(True)
+    run_steps(args.steps)
+    torch.cuda.synchronize()
+    kt = rapi.rpa_get_kernel_timing()
+    rapi.rpa_set_kernel_timing(False)
+    busy_ms = sum(block_ms)
 
     def kernel_roofline(kind):
         total_ms, launches = kt[kind]
@@ -389,22 +382,25 @@ def main():
         k_ms = total_ms / launches
         if kind == "tile":  # dense contractions on the tensor cores
             achieved = info["tile_flops"] / 1e12 / (k_ms * 1e-3)
-            peak = float(peaks["bf16_tflops"] if timed_ms < 2000 else peaks["bf16_tflops_sustained"])
+            # the cuBLAS burst figure: the larger (stricter) denominator; the sustained one is given beside it
+            peak = float(peaks["bf16_tflops"])
             kbound, runit, nominal = "tensor", "TFLOP/s", NOMINAL_BF16_TFLOPS
         else:  # the split-KV row kernel streams the cache: HBM
             achieved = info["row_bytes"] / 1e9 / (k_ms * 1e-3)
             peak, kbound, runit, nominal = float(peaks["hbm_gbs"]), "hbm", "GB/s", NOMINAL_HBM_GBS
-        return {"bound": kbound, "kernel": f"rpa_{kind}_kernel", "achieved": achieved, "peak": peak, "unit": runit,
-                "frac": achieved / peak, "peak_source": peaks["_source"], "traffic": None, "kernel_ms": k_ms,
-                "kernel_launches": launches, "kernel_share_of_step": total_ms / max(1e-9, timed_ms),
-                "frac_of_nominal": achieved / nominal}
+        r = {"bound": kbound, "kernel": f"rpa_{kind}_kernel", "achieved": achieved, "peak": peak, "unit": runit,
+             "frac": achieved / peak, "peak_source": peaks["_source"], "traffic": None, "kernel_ms": k_ms,
+             "kernel_launches": launches, "kernel_share_of_step": k_ms / max(1e-9, ms_per_step),
+             "frac_of_nominal": achieved / nominal}
+        if kind == "tile":
+            r["frac_of_sustained_peak"] = achieved / float(peaks["bf16_tflops_sustained"])
+        return r
 
-    timed_ms = e0.elapsed_time(e1)
     dom = max(("row", "tile", "combine"), key=lambda k: kt[k][0])
     roofline = kernel_roofline(dom)
     other = [kernel_roofline(k) for k in ("row", "tile") if k != dom and kt[k][1] > 0]
-    traffic_key = (args.workload, dom, bool(meta.kv_fp8))
-    if traffic_key in NCU_TRAFFIC and rank == 0 and meta.seed == 1000 + cfg and args.plan == "host":
+    traffic_key = (workload, dom, bool(meta.kv_fp8))
+    if roofline and traffic_key in NCU_TRAFFIC and rank == 0 and meta.seed == 1000 + (4 if cfg == "4b" else cfg) and args.plan == "host":
         roofline["traffic"], roofline["traffic_source"] = NCU_TRAFFIC[traffic_key]
 
     # ---- end to end: host buffers through rpa_forward_host, copies inside the timed region ----
@@ -427,30 +423,21 @@ def main():
                     rapi.rpa_forward_host_wait()
             rapi.rpa_forward_host_wait()
 
+        def e2e_serial(k):  # one at a time: rpa_forward_host returns with the output on the host
+            for i in range(k):
+                rapi.rpa_forward_host(hq, hk, hv, batch.kv_cache, hpt, hcu, hkl, houts[i & 1], sh)
+
         e2e_steps(3)
-        if dist:
-            dist.barrier()
-        torch.cuda.synchronize()
-        e0.record(stream)
-        e2e_steps(args.steps)  # returns when the last step's output has reached the host
-        e1.record(stream)
-        torch.cuda.synchronize()
-        ms_e2e, _ = aggregate_over_ranks(e0.elapsed_time(e1), 0.0, dist, torch.device("cuda", local))
-        # for comparison: the same steps one at a time (rpa_forward_host returns with the output on the host)
+        ms_e2e = median(timed_blocks(e2e_steps, args.steps, 0.5 * args.min_seconds, dist, device, max_blocks=400)) / args.steps
         n_serial = max(3, args.steps // 4)
-        e0.record(stream)
-        for i in range(n_serial):
-            rapi.rpa_forward_host(hq, hk, hv, batch.kv_cache, hpt, hcu, hkl, houts[i & 1], sh)
-        e1.record(stream)
-        torch.cuda.synchronize()
-        ms_serial, _ = aggregate_over_ranks(e0.elapsed_time(e1), 0.0, dist, torch.device("cuda", local))
+        ms_serial = median(timed_blocks(e2e_serial, n_serial, 0.25 * args.min_seconds, dist, device, max_blocks=400)) / n_serial
         row_q = meta.num_q_heads * meta.head_dim * 2
         row_k = meta.num_kv_heads * meta.head_dim * 2
         h2d = T * (row_q + 2 * row_k) + n * meta.max_pages_per_seq * 4 + (2 * n + 1) * 4 + info["num_row_items"] * 32
-        e2e = {"value": units_per_step / (ms_e2e / args.steps * 1e-3), "unit": unit, "h2d_bytes_per_step": int(h2d),
-               "d2h_bytes_per_step": int(T * row_q), "ms_per_step": ms_e2e / args.steps,
+        e2e = {"value": units_per_step / (ms_e2e * 1e-3), "unit": unit, "h2d_bytes_per_step": int(h2d),
+               "d2h_bytes_per_step": int(T * row_q), "ms_per_step": ms_e2e,
                "steps_in_flight": 2,
-               "one_step_in_flight": {"value": units_per_step / (ms_serial / n_serial * 1e-3), "ms_per_step": ms_serial / n_serial,
+               "one_step_in_flight": {"value": units_per_step / (ms_serial * 1e-3), "ms_per_step": ms_serial,
                                       "steps": n_serial},
                "note": "rpa_forward_host_submit / rpa_forward_host_wait, two steps in flight: every step copies its "
                        "inputs from pinned host memory and its output back; the KV cache stays resident in HBM"}
@@ -458,42 +445,161 @@ def main():
     # ---- CPU baseline: the oracle on a bounded sample, rank 0 at N=1 only ----
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        dt, units, what, cores = oracle_sample(meta, batch, budget_s=15.0)
+        dt, units, what, cores = oracle_sample(meta, batch, budget_s=args.cpu_budget)
         cpu_baseline = {"value": units[unit_key(unit)] / dt, "unit": unit, "cores": cores, "kind": "oracle",
                         "sample": what, "seconds": dt}
 
+    rapi.close()
+    launches_per_step = device_plan_launches(meta) if args.plan == "device" else info["gpu_launches"]
+    return {
+        "metric": metric, "value": value, "unit": unit, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+        "scaling": "strong" if (args.shard == "heads" and world > 1) else "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": meta.name, "kv_cache": "fp8_e4m3" if meta.kv_fp8 else "bf16",
+                   "num_seqs": meta.num_seqs, "num_tokens": meta.num_tokens,
+                   "kv_tokens": int(meta.kv_lens.sum()), "heads": f"{meta.num_q_heads}q/{meta.num_kv_heads}kv",
+                   "head_dim": meta.head_dim, "page_size": meta.page_size, "num_pages": meta.num_pages,
+                   "causal": bool(meta.causal), "batch_case": info["batch_case_name"], "row_items": info["num_row_items"],
+                   "tile_items": info["num_tile_items"], "combine_groups": info["num_combine_groups"],
+                   "kv_chunk_tokens": info["kv_chunk_tokens"], "parallelism": (f"tp{world}" if args.shard == "heads" and world > 1 else f"dp{world}"),
+                   "step": ("rpa_plan_device (for the next step, on a side stream)" if args.plan == "device" else "rpa_plan") + " + rpa_forward",
+                   "l2": ("KV working set %.2f GB per step exceeds the 126 MB L2; no flush needed" % (info["algorithmic_bytes"] / 1e9))
+                         if bound == "hbm" else "compute-bound: K/V re-reads through L2 are part of the method; no flush"},
+        "timing": {"blocks": len(block_ms), "steps_per_block": args.steps, "gpu_seconds_timed": busy_ms * 1e-3,
+                   "block_ms_median": median(block_ms), "block_ms_min": min(block_ms), "block_ms_max": max(block_ms),
+                   "per_kernel_events_in_timed_blocks": False},
+        "clocks": clocks.summary(),
+        "roofline": roofline,
+        "roofline_other_kernels": other,
+        "e2e": e2e,
+        "cpu_baseline": cpu_baseline,
+        # device-planned steps always launch the plan kernel and every attention kernel the handle
+        # may need: with an FP8 cache the 8-row and the 16-row instantiation of the row kernel (when
+        # there are at most 8 grouped heads) and the quantising pass before the tile kernel
+        "gpu_launches": args.steps * launches_per_step,
+        "gpu_launches_per_step": launches_per_step,
+        "mbu_vs_nominal_8TBs": value / NOMINAL_HBM_GBS / world if unit == "GB/s" else None,
+        "mfu_vs_nominal_2250": value / NOMINAL_BF16_TFLOPS / world if unit == "TFLOP/s" else None,
+        "achieved_gbs": info["algorithmic_bytes"] / 1e9 / (ms_per_step * 1e-3),
+        "achieved_tflops": info["algorithmic_flops"] / 1e12 / (ms_per_step * 1e-3),
+    }
+
+
+def run_plan_only(args):
+    """No device: every rank plans its shard of the headline batch on the host (gloo for the
+    aggregation) and rank 0 prints what the launch would cover.  Exercises the launch plumbing of
+    ``--gpus N`` on a machine without GPUs; no throughput is reported."""
+    from paper_2604_15464_b200 import binding, build
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+
+        dist.init_process_group("gloo")
+    if rank == 0:
+        build.build()
+    if dist:
+        dist.barrier()
+    workload = "decode" if args.workload == "all" else args.workload
+    meta = wl.workload_meta(WORKLOADS[workload][0], seed=1000 + 2 + 7919 * rank) if workload == "decode" else make_meta(workload, rank, 1.0, args)
+    rapi = binding.Rpa.for_meta(meta, device=-1)
+    rapi.rpa_plan(meta.cu_q_lens, meta.kv_lens)
+    info = rapi.rpa_plan_info()
+    _, units = aggregate_over_ranks(0.0, units_of(workload, info, meta), dist, torch.device("cpu"))
+    if rank == 0:
+        print(json.dumps({"plan_only": True, "metric": WORKLOADS[workload][1], "value": None, "unit": WORKLOADS[workload][2],
+                          "n_gpus": world, "units_per_step": units, "config": {"workload": meta.name}}))
+    if dist:
+        dist.destroy_process_group()
+    return 0
+
+
+def respawn_under_torchrun(args) -> int:
+    """``--gpus N`` outside a torchrun environment: start N ranks of this script, one per GPU."""
+    import socket
+
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__), *sys.argv[1:]]
+    return subprocess.call(cmd)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="all", choices=sorted(WORKLOADS) + ["all"],
+                    help="all: the decode batch as the headline line with the prefill and mixed batches under \"legs\"")
+    ap.add_argument("--min-seconds", type=float, default=1.0,
+                    help="blocks of --steps steps are repeated until this much GPU time has been timed; the median block is reported")
+    ap.add_argument("--cpu-budget", type=float, default=12.0, help="seconds of CPU work the oracle sample of each leg is sized for")
+    ap.add_argument("--pool-gb", type=float, default=None, help="cache pool size for the skewed workload")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--plan-only", action="store_true", help="no device: plan the headline batch on every rank and print the launch's shape")
+    ap.add_argument("--kv-chunk", type=int, default=0)
+    ap.add_argument("--ablate", type=int, default=0, help="rpa_set_ablation mask (1: no cache update, 2: no kernel overlap, 4: no attention arithmetic, 8: no K/V loads)")
+    ap.add_argument("--ctx", type=int, default=8192, help="context length of the paper_decode workload")
+    ap.add_argument("--seq", type=int, default=8192, help="sequence length of the paper_prefill workload")
+    ap.add_argument("--paper-n", type=int, default=0, help="requests in the paper_* workloads (default 128 / 1)")
+    ap.add_argument("--page-size", type=int, default=256, help="page size of the paper_* workloads")
+    ap.add_argument("--noncausal", action="store_true", help="paper_* workloads without the causal mask")
+    ap.add_argument("--head-dim", type=int, default=128, help="head dimension of the paper_* workloads (128 or 256)")
+    ap.add_argument("--kv-fp8", action="store_true", help="FP8 E4M3 cache with per-tensor scales (decode workloads)")
+    ap.add_argument("--plan", default="host", choices=["host", "device"],
+                    help="who builds the work lists each step: rpa_plan on the host, or rpa_plan_device on the GPU")
+    ap.add_argument("--shard", default="requests", choices=["requests", "heads"],
+                    help="how N ranks split the work: own requests each (weak scaling) or own KV heads each (strong)")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        return respawn_under_torchrun(args)
+    if args.impl == "reference":
+        if args.workload == "all":
+            args.workload = "decode"
+        return run_reference(args)
+    if args.plan_only:
+        return run_plan_only(args)
+
+    from paper_2604_15464_b200 import binding, build
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the product has no CPU path")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    if rank == 0:
+        build.build()
+    if dist:
+        dist.barrier()
+    binding.load_library()
+    peaks = load_peaks()
+
+    names = ["decode", "prefill", "mixed"] if args.workload == "all" else [args.workload]
+    line = run_leg(names[0], args, rank, world, local, dist, peaks)
+    if len(names) > 1:
+        line["legs"] = {}
+        for name in names[1:]:
+            torch.cuda.empty_cache()
+            line["legs"][name] = run_leg(name, args, rank, world, local, dist, peaks)
+        line["gpu_launches_all_legs"] = line["gpu_launches"] + sum(l["gpu_launches"] for l in line["legs"].values())
     if dist:
         dist.barrier()
     if rank == 0:
-        line = {
-            "metric": metric, "value": value, "unit": unit, "n_gpus": world, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
-            "scaling": "strong" if (args.shard == "heads" and world > 1) else "weak",
-            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": meta.name, "kv_cache": "fp8_e4m3" if meta.kv_fp8 else "bf16",
-                       "num_seqs": meta.num_seqs, "num_tokens": meta.num_tokens,
-                       "kv_tokens": int(meta.kv_lens.sum()), "heads": f"{meta.num_q_heads}q/{meta.num_kv_heads}kv",
-                       "head_dim": meta.head_dim, "page_size": meta.page_size, "num_pages": meta.num_pages,
-                       "causal": bool(meta.causal), "batch_case": info["batch_case_name"], "row_items": info["num_row_items"],
-                       "tile_items": info["num_tile_items"], "combine_groups": info["num_combine_groups"],
-                       "kv_chunk_tokens": info["kv_chunk_tokens"], "parallelism": (f"tp{world}" if args.shard == "heads" and world > 1 else f"dp{world}"),
-                       "step": ("rpa_plan_device (for the next step, on a side stream)" if args.plan == "device" else "rpa_plan") + " + rpa_forward",
-                       "l2": "KV working set %.2f GB per step exceeds the 126 MB L2; no flush needed"
-                             % (info["algorithmic_bytes"] / 1e9)},
-            "clocks": clocks.summary(),
-            "roofline": roofline,
-            "roofline_other_kernels": other,
-            "e2e": e2e,
-            "cpu_baseline": cpu_baseline,
-            # device-planned steps always launch the plan kernel and every attention kernel the handle
-            # may need: with an FP8 cache the 8-row and the 16-row instantiation of the row kernel (when
-            # there are at most 8 grouped heads) and the quantising pass before the tile kernel
-            "gpu_launches": args.steps * (device_plan_launches(meta) if args.plan == "device" else info["gpu_launches"]),
-            "mbu_vs_nominal_8TBs": value / NOMINAL_HBM_GBS / world if unit == "GB/s" else None,
-            "mfu_vs_nominal_2250": value / NOMINAL_BF16_TFLOPS / world if unit == "TFLOP/s" else None,
-            "achieved_gbs": info["algorithmic_bytes"] / 1e9 / (ms_per_step * 1e-3),
-            "achieved_tflops": info["algorithmic_flops"] / 1e12 / (ms_per_step * 1e-3),
-        }
         print(json.dumps(line))
     if dist:
         dist.destroy_process_group()

@@ -79,3 +79,26 @@ def test_head_sharding_splits_the_work_without_overlap():
     assert sum(p["algorithmic_flops"] for p in parts) == whole["algorithmic_flops"]
     with pytest.raises(ValueError):
         bench.shard_heads(wl.workload_meta(2), 0, 3)
+
+
+def test_bench_gpus_n_starts_n_ranks_by_itself():
+    """``python bench.py --gpus 2`` outside a torchrun environment must start two ranks (it re-executes
+    itself under torch.distributed.run); checked here without a device through the planning-only
+    mode, in which the ranks meet over gloo and rank 0 reports the size of the job."""
+    import json
+    import subprocess
+
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    res = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--plan-only"], env=env,
+                         capture_output=True, text=True, timeout=600)
+    assert res.returncode == 0, res.stderr[-2000:]
+    lines = [l for l in res.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1  # rank 0 alone prints
+    line = json.loads(lines[0])
+    assert line["n_gpus"] == 2 and line["plan_only"] is True
+    # two different batches of the decode shape: about twice one batch's bytes
+    one = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--plan-only"], env=env, capture_output=True,
+                         text=True, timeout=600)
+    single = json.loads([l for l in one.stdout.splitlines() if l.startswith("{")][0])
+    assert single["n_gpus"] == 1
+    assert 1.7 * single["units_per_step"] < line["units_per_step"] < 2.3 * single["units_per_step"]
