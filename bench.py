@@ -184,15 +184,16 @@ def units_of(workload: str, info: dict, meta) -> float:
     return float(meta.num_tokens)  # tokens
 
 
-def oracle_sample(meta, batch, budget_s: float = 15.0):
-    """Times the CPU oracle, as it stands, on a bounded sample of the batch's requests.  Returns
-    (seconds, units-dict of the sample, description)."""
+def oracle_sample(meta, batch, budget_s: float = 15.0, rate: float | None = None):
+    """Times the CPU oracle, as it stands, on a bounded sample of the batch's requests.  ``rate`` is
+    the oracle's speed (nominal FLOP/s over all cores) used to size the sample; the time is measured.
+    Returns (seconds, units-dict of the sample, description, cores, nominal FLOPs of the sample)."""
     from oracle import rpa_oracle as orc  # CPU-baseline leg only
 
-    order = np.argsort(-(meta.kv_lens.astype(np.int64) * np.maximum(meta.q_lens, 0)))
     cost = meta.q_lens.astype(np.float64) * meta.kv_lens * meta.num_q_heads * meta.head_dim * 4  # ~flops
     cores = orc.threads()
-    rate = 0.35e9 * cores  # conservative fp64 scalar rate to size the sample; the time is measured
+    if rate is None:
+        rate = 0.35e9 * cores  # conservative fp64 scalar rate for a first, short sample
     pick, acc = [], 0.0
     for r in np.random.default_rng(5).permutation(meta.num_seqs):
         if meta.q_lens[r] == 0:
@@ -228,8 +229,20 @@ def oracle_sample(meta, batch, budget_s: float = 15.0):
         "TFLOP": frac * metrics.attention_flops(ql, kl, meta.num_q_heads, meta.head_dim, meta.causal) / 1e12,
         "tokens": frac * float(ql.sum()),
     }
+    n_live = int((meta.q_lens > 0).sum())
+    whole = len(pick) == n_live and frac == 1.0
     what = f"{len(pick)} of {meta.num_seqs} requests" + (f", {len(triples)} sampled (token, head) rows" if frac < 1 else ", all rows")
-    return dt, units, what, cores
+    return dt, units, what, cores, (frac * acc, whole)
+
+
+def cpu_baseline_of(meta, batch, unit, budget_s):
+    """The oracle on a sample sized for about ``budget_s`` seconds of CPU work: a first short sample
+    measures its speed on this machine and this workload, a second one is sized with that speed (unless
+    the first already covered the whole batch)."""
+    dt, units, what, cores, (flops, whole) = oracle_sample(meta, batch, budget_s=min(budget_s, 3.0))
+    if not whole and dt < 0.6 * budget_s:
+        dt, units, what, cores, _ = oracle_sample(meta, batch, budget_s=budget_s, rate=max(flops / max(dt, 1e-3), 1e6))
+    return {"value": units[unit_key(unit)] / dt, "unit": unit, "cores": cores, "kind": "oracle", "sample": what, "seconds": dt}
 
 
 def unit_key(unit: str) -> str:
@@ -247,10 +260,12 @@ def run_reference(args):
     else:
         meta = wl.workload_meta(cfg, num_pages=None if cfg != 5 else 40000)
     batch = wl.materialize(meta, "cpu")
-    times, total_units, what, cores = [], 0.0, "", 1
+    times, total_units, what, cores, rate = [], 0.0, "", 1, None
     budget = max(2.0, min(20.0, 90.0 / max(1, args.steps + args.warmup)))
     for step in range(args.warmup + args.steps):
-        dt, units, what, cores = oracle_sample(meta, batch, budget_s=budget)
+        dt, units, what, cores, (flops, _) = oracle_sample(meta, batch, budget_s=budget, rate=rate)
+        if step == 0 and args.warmup > 0:  # the first warm-up sample calibrates the size of the later ones
+            rate = max(flops / max(dt, 1e-3), 1e6)
         if step >= args.warmup:
             times.append(dt)
             total_units += units[unit_key(unit)]
@@ -445,9 +460,7 @@ def run_leg(workload, args, rank, world, local, dist, peaks):
     # ---- CPU baseline: the oracle on a bounded sample, rank 0 at N=1 only ----
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        dt, units, what, cores = oracle_sample(meta, batch, budget_s=args.cpu_budget)
-        cpu_baseline = {"value": units[unit_key(unit)] / dt, "unit": unit, "cores": cores, "kind": "oracle",
-                        "sample": what, "seconds": dt}
+        cpu_baseline = cpu_baseline_of(meta, batch, unit, args.cpu_budget)
 
     rapi.close()
     launches_per_step = device_plan_launches(meta) if args.plan == "device" else info["gpu_launches"]

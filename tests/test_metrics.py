@@ -74,7 +74,7 @@ def test_bench_cpu_baseline_leg_runs_on_bf16_and_fp8_caches():
         meta = wl.build_meta("cpu_leg", [1, 5, 1], [40, 5, 130], num_q_heads=8, num_kv_heads=2, head_dim=64, page_size=16,
                              seed=3, **extra)
         batch = wl.materialize(meta, torch.device("cpu"))
-        dt, units, what, cores = bench.oracle_sample(meta, batch, budget_s=1.0)
+        dt, units, what, cores, _ = bench.oracle_sample(meta, batch, budget_s=1.0)
         assert dt > 0 and cores >= 1 and what.startswith("3 of 3 requests")
         assert units["tokens"] == 7
         kv_bytes = 1 if fp8 else 2
