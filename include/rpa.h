@@ -43,7 +43,9 @@
  *
  * Ownership: the caller owns every tensor and the stream.  The handle owns the plan (device work
  * lists) and the split-KV workspace, both allocated in rpa_create from the capacities in
- * rpa_config_t; rpa_plan and rpa_forward allocate nothing.  kv_cache is updated in place; out rows
+ * rpa_config_t; rpa_plan and rpa_forward allocate nothing.  Two optional paths allocate once more,
+ * on their first use: rpa_forward_host_submit / rpa_forward_host (two sets of staging buffers for
+ * the step's tensors) and rpa_plan_device (its own lists and scratch).  kv_cache is updated in place; out rows
  * >= T and every cache slot other than the T*h_kv updated ones are left bit-identical.
  *
  * Preconditions (undefined behaviour otherwise): page ids lie in [0, num_pages); pages holding
@@ -135,11 +137,14 @@ void rpa_destroy(rpa_handle_t* h);
  * cu_q_lens_host [n+1] and kv_lens_host [n] are HOST pointers.  Classifies every sequence (decode
  * q_r == 1, prefill q_r > 1) and the batch, builds the work lists (split-KV chunks for the row
  * kernel, query tiles for the tile kernel, combine groups, one designated cache writer per new
- * token and KV head) and starts their copy to the device on a stream the handle owns, into the one
- * of two list buffers that the previous plan does not use: planning step i+1 never waits for the
- * kernels of step i.  rpa_forward orders itself after the copy.  `stream` is reserved (pass the
- * stream the next rpa_forward will use, or null).  Does not wait for the copy.  A plan stays valid
- * for any number of rpa_forward calls with the same lengths.
+ * token and KV head) and starts their copy to the device (one copy of one packed block: the lists,
+ * then the lengths) on a stream the handle owns, into the next of a ring of four list buffers:
+ * planning step i+1 never waits for the kernels of step i.  rpa_forward orders itself after the
+ * copy.  `stream` is reserved (pass the stream the next rpa_forward will use, or null).  Does not
+ * wait for the copy, and does not wait for the device at all unless the caller is four plans ahead
+ * of it (the pinned mirror of the buffer it is about to fill then still feeds the copy of the plan
+ * made four calls ago; a loop that enqueues steps without ever synchronising is throttled to that
+ * depth).  A plan stays valid for any number of rpa_forward calls with the same lengths.
  */
 rpa_status_t rpa_plan(rpa_handle_t* h, const int32_t* cu_q_lens_host, const int32_t* kv_lens_host,
                       int32_t num_seqs, void* stream);
@@ -168,7 +173,8 @@ rpa_status_t rpa_forward_host(rpa_handle_t* h, const void* q_host, const void* n
 /*
  * The two halves of rpa_forward_host, for callers that keep more than one step in flight.
  * rpa_forward_host_submit takes the same arguments, plans on the calling thread, enqueues the
- * input copies on a copy stream of the handle, the kernels on `stream` and the output copy on a
+ * input copies (q, new_k, new_v and the page table; the lengths travel with the plan's lists) on a
+ * copy stream of the handle, the kernels on `stream` and the output copy on a
  * second copy stream, and returns without waiting: the copies of a step run beside the kernels of
  * its neighbours (two sets of staging buffers; a third outstanding step waits, on the device, for
  * the first one's output copy).  Steps run in submission order on `stream`, so each sees the cache

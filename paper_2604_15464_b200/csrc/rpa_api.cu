@@ -26,20 +26,26 @@ struct rpa_handle {
     uint32_t ablation = 0;
     std::string last_error;
 
-    // Device work lists, [row items | tile items | combine groups], double-buffered so that the
-    // copy of the next plan (on an internal stream) overlaps the kernels of the current one.
-    uint8_t* d_lists[2] = {nullptr, nullptr};
-    uint8_t* h_lists[2] = {nullptr, nullptr};  // pinned mirrors
+    // Device work lists, [row items | tile items | combine groups | kv_lens | cu_q_lens], in a ring of
+    // kPlanRing buffers so that the copy of the next plans (on an internal stream) overlaps the kernels
+    // of the current one.  A host-made plan is packed tightly (the offsets of its sections are kept per
+    // buffer) and travels in one copy; off_tiles / off_groups / off_kvlens are the offsets at full
+    // capacity, used for the buffers' size and by the device-side planner.
+    static constexpr int kPlanRing = 4;
+    uint8_t* d_lists[kPlanRing] = {};
+    uint8_t* h_lists[kPlanRing] = {};  // pinned mirrors
+    size_t buf_off_tiles[kPlanRing] = {}, buf_off_groups[kPlanRing] = {}, buf_off_kvlens[kPlanRing] = {}, buf_off_cu[kPlanRing] = {};
     size_t off_tiles = 0, off_groups = 0, lists_bytes = 0;
+    TileMapCache tile_maps;  // tensor maps of the tile kernels, keyed by the tensors they describe
     cudaStream_t copy_stream = nullptr;
     cudaStream_t aux_stream = nullptr;  // the tile kernel of a mixed batch runs here, beside the row kernel
     cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
     cudaStream_t aux2_stream = nullptr;  // device-planned FP8 steps: the row kernel instantiation the list may not need
     cudaEvent_t ev_fork2 = nullptr, ev_join2 = nullptr;
-    cudaEvent_t ev_copied[2] = {nullptr, nullptr};    // plan copy into buffer b finished
-    cudaEvent_t ev_consumed[2] = {nullptr, nullptr};  // last forward that read buffer b finished
-    bool copied_pending[2] = {false, false};
-    bool consumed_pending[2] = {false, false};
+    cudaEvent_t ev_copied[kPlanRing] = {};    // plan copy into buffer b finished
+    cudaEvent_t ev_consumed[kPlanRing] = {};  // last forward that read buffer b finished
+    bool copied_pending[kPlanRing] = {};
+    bool consumed_pending[kPlanRing] = {};
     int cur = 0;  // buffer holding the current plan
     bool validate = false;        // run the input validation kernel before the attention kernels
     size_t off_kvlens = 0;        // the plan's kv_lens travel with the lists (for the validation kernel)
@@ -110,7 +116,7 @@ bool valid_config(const rpa_config_t& c, rpa_status_t* why) {
 
 void free_all(rpa_handle* h) {
     if (!h->plan_only) {
-        for (int b = 0; b < 2; ++b) {
+        for (int b = 0; b < rpa_handle::kPlanRing; ++b) {
             cudaFree(h->d_lists[b]);
             if (h->h_lists[b]) cudaFreeHost(h->h_lists[b]);
             if (h->ev_copied[b]) cudaEventDestroy(h->ev_copied[b]);
@@ -252,7 +258,8 @@ rpa_status_t rpa_create(const rpa_config_t* cfg, int device, rpa_handle_t** out)
     h->off_tiles = align_up((size_t)p.max_row_items * sizeof(RowItem), 256);
     h->off_groups = h->off_tiles + align_up((size_t)std::max(p.max_tile_items, 1) * sizeof(TileItem), 256);
     h->off_kvlens = h->off_groups + align_up((size_t)p.max_groups * sizeof(CombineGroup), 256);
-    h->lists_bytes = h->off_kvlens + align_up((size_t)cfg->max_num_seqs * sizeof(int32_t), 256);
+    h->lists_bytes = h->off_kvlens + align_up((size_t)cfg->max_num_seqs * sizeof(int32_t), 256) +
+                     align_up(((size_t)cfg->max_num_seqs + 1) * sizeof(int32_t), 256);
 
     if (!h->plan_only) {
         cudaError_t e = cudaStreamCreateWithFlags(&h->copy_stream, cudaStreamNonBlocking);
@@ -264,7 +271,7 @@ rpa_status_t rpa_create(const rpa_config_t* cfg, int device, rpa_handle_t** out)
         if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&h->aux2_stream, cudaStreamNonBlocking);
         if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_fork2, cudaEventDisableTiming);
         if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_join2, cudaEventDisableTiming);
-        for (int b = 0; b < 2 && e == cudaSuccess; ++b) {
+        for (int b = 0; b < rpa_handle::kPlanRing && e == cudaSuccess; ++b) {
             e = cudaMalloc(&h->d_lists[b], h->lists_bytes);
             if (e == cudaSuccess) e = cudaMallocHost(&h->h_lists[b], h->lists_bytes);
             if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_copied[b], cudaEventDisableTiming);
@@ -305,39 +312,36 @@ rpa_status_t rpa_plan(rpa_handle_t* h, const int32_t* cu_q_lens_host, const int3
     if (!h->plan_only) {
         st = ensure_device(h);
         if (st != RPA_OK) return st;
-        // The copy goes into the buffer the current plan does not use, on the internal stream: it
-        // may run while the kernels of the previous rpa_forward are still in flight.
-        const int b = h->cur ^ 1;
-        if (h->copied_pending[b]) {  // the pinned mirror may still feed an older copy
-            RPA_CUDA(h, cudaEventSynchronize(h->ev_copied[b]));
+        // The copy goes into the next buffer of the ring, on the internal stream: it may run while the
+        // kernels of earlier rpa_forward calls are still in flight.  The host waits only if the pinned
+        // mirror of that buffer still feeds the copy of the plan made kPlanRing calls ago (the caller is
+        // that many plans ahead of the device).
+        const int b = (h->cur + 1) % rpa_handle::kPlanRing;
+        if (h->copied_pending[b]) {
+            if (cudaEventQuery(h->ev_copied[b]) != cudaSuccess) RPA_CUDA(h, cudaEventSynchronize(h->ev_copied[b]));
             h->copied_pending[b] = false;
         }
         if (h->consumed_pending[b]) {  // kernels of an older rpa_forward may still read the device buffer
             RPA_CUDA(h, cudaStreamWaitEvent(h->copy_stream, h->ev_consumed[b], 0));
             h->consumed_pending[b] = false;
         }
+        // one tightly packed block, one copy: [row items | tile items | groups | kv_lens | cu_q_lens]
         const size_t nb_rows = h->plan.rows.size() * sizeof(RowItem);
         const size_t nb_tiles = h->plan.tiles.size() * sizeof(TileItem);
         const size_t nb_groups = h->plan.groups.size() * sizeof(CombineGroup);
-        if (nb_rows) {
-            memcpy(h->h_lists[b], h->plan.rows.data(), nb_rows);
-            RPA_CUDA(h, cudaMemcpyAsync(h->d_lists[b], h->h_lists[b], nb_rows, cudaMemcpyHostToDevice, h->copy_stream));
-        }
-        if (nb_tiles) {
-            memcpy(h->h_lists[b] + h->off_tiles, h->plan.tiles.data(), nb_tiles);
-            RPA_CUDA(h, cudaMemcpyAsync(h->d_lists[b] + h->off_tiles, h->h_lists[b] + h->off_tiles, nb_tiles,
-                                        cudaMemcpyHostToDevice, h->copy_stream));
-        }
-        if (nb_groups) {
-            memcpy(h->h_lists[b] + h->off_groups, h->plan.groups.data(), nb_groups);
-            RPA_CUDA(h, cudaMemcpyAsync(h->d_lists[b] + h->off_groups, h->h_lists[b] + h->off_groups, nb_groups,
-                                        cudaMemcpyHostToDevice, h->copy_stream));
-        }
-        if (num_seqs > 0) {
-            memcpy(h->h_lists[b] + h->off_kvlens, kv_lens_host, (size_t)num_seqs * sizeof(int32_t));
-            RPA_CUDA(h, cudaMemcpyAsync(h->d_lists[b] + h->off_kvlens, h->h_lists[b] + h->off_kvlens,
-                                        (size_t)num_seqs * sizeof(int32_t), cudaMemcpyHostToDevice, h->copy_stream));
-        }
+        const size_t n = (size_t)std::max(num_seqs, 0);
+        h->buf_off_tiles[b] = align_up(nb_rows, 256);
+        h->buf_off_groups[b] = h->buf_off_tiles[b] + align_up(nb_tiles, 256);
+        h->buf_off_kvlens[b] = h->buf_off_groups[b] + align_up(nb_groups, 256);
+        h->buf_off_cu[b] = h->buf_off_kvlens[b] + align_up(n * sizeof(int32_t), 256);
+        const size_t total = h->buf_off_cu[b] + (n + 1) * sizeof(int32_t);
+        uint8_t* m = h->h_lists[b];
+        if (nb_rows) memcpy(m, h->plan.rows.data(), nb_rows);
+        if (nb_tiles) memcpy(m + h->buf_off_tiles[b], h->plan.tiles.data(), nb_tiles);
+        if (nb_groups) memcpy(m + h->buf_off_groups[b], h->plan.groups.data(), nb_groups);
+        if (n) memcpy(m + h->buf_off_kvlens[b], kv_lens_host, n * sizeof(int32_t));
+        if (n) memcpy(m + h->buf_off_cu[b], cu_q_lens_host, (n + 1) * sizeof(int32_t));
+        RPA_CUDA(h, cudaMemcpyAsync(h->d_lists[b], m, total, cudaMemcpyHostToDevice, h->copy_stream));
         RPA_CUDA(h, cudaEventRecord(h->ev_copied[b], h->copy_stream));
         h->copied_pending[b] = true;
         h->cur = b;
@@ -348,7 +352,7 @@ rpa_status_t rpa_plan(rpa_handle_t* h, const int32_t* cu_q_lens_host, const int3
 
 // The kernel arguments every launch of a call shares: tensors, shape, scales; `lists` is the device
 // buffer holding [row items | tile items | combine groups].  Counts are filled in by the caller.
-static KernelArgs common_kernel_args(const rpa_handle* h, uint8_t* lists, const void* q, const void* new_k, const void* new_v,
+static KernelArgs common_kernel_args(const rpa_handle* h, uint8_t* lists, size_t off_tiles, size_t off_groups, const void* q, const void* new_k, const void* new_v,
                                      void* kv_cache, const int32_t* page_table, const int32_t* cu_q_lens,
                                      const int32_t* kv_lens, void* out) {
     const rpa_config_t& c = h->cfg;
@@ -364,8 +368,8 @@ static KernelArgs common_kernel_args(const rpa_handle* h, uint8_t* lists, const 
     a.kv_lens = kv_lens;
     a.out = static_cast<uint16_t*>(out);
     a.row_items = reinterpret_cast<const RowItem*>(lists);
-    a.tile_items = reinterpret_cast<const TileItem*>(lists + h->off_tiles);
-    a.groups = reinterpret_cast<const CombineGroup*>(lists + h->off_groups);
+    a.tile_items = reinterpret_cast<const TileItem*>(lists + off_tiles);
+    a.groups = reinterpret_cast<const CombineGroup*>(lists + off_groups);
     a.partial_o = h->d_partial_o;
     a.partial_ml = h->d_partial_ml;
     a.status = h->d_status;
@@ -399,7 +403,7 @@ static rpa_status_t forward_device_planned(rpa_handle* h, const void* q, const v
     if (!aligned16(q) || !aligned16(new_k) || !aligned16(new_v) || !aligned16(kv_cache) || !aligned16(out))
         return RPA_ERR_INVALID_ARG;
     const rpa_config_t& c = h->cfg;
-    KernelArgs a = common_kernel_args(h, h->d_dev_lists, q, new_k, new_v, kv_cache, page_table, cu_q_lens, kv_lens, out);
+    KernelArgs a = common_kernel_args(h, h->d_dev_lists, h->off_tiles, h->off_groups, q, new_k, new_v, kv_cache, page_table, cu_q_lens, kv_lens, out);
     a.group_counters = h->d_group_counters;
     a.dev_counts = h->d_dev_counts;
     a.num_tile_ctas = h->num_sms;
@@ -415,8 +419,8 @@ static rpa_status_t forward_device_planned(rpa_handle* h, const void* q, const v
         RPA_CUDA(h, cudaStreamWaitEvent(h->aux_stream, h->ev_fork, 0));
         const bool single_tile = tile1_kernel_supported(c.head_dim, c.num_q_heads / c.num_kv_heads);
         timing_mark(h, 1, h->aux_stream);
-        RPA_CUDA(h, single_tile ? launch_tile1_kernel(a, c.max_num_tokens, h->aux_stream)
-                                : launch_tile_kernel(a, c.max_num_tokens, h->aux_stream));
+        RPA_CUDA(h, single_tile ? launch_tile1_kernel(a, c.max_num_tokens, &h->tile_maps, h->aux_stream)
+                                : launch_tile_kernel(a, c.max_num_tokens, &h->tile_maps, h->aux_stream));
         timing_mark(h, 1, h->aux_stream);
         RPA_CUDA(h, cudaEventRecord(h->ev_join, h->aux_stream));
     }
@@ -581,7 +585,8 @@ rpa_status_t rpa_forward(rpa_handle_t* h, const void* q, const void* new_k, cons
     if (st != RPA_OK) return st;
 
     uint8_t* lists = h->d_lists[h->cur];
-    KernelArgs a = common_kernel_args(h, lists, q, new_k, new_v, kv_cache, page_table, cu_q_lens, kv_lens, out);
+    KernelArgs a = common_kernel_args(h, lists, h->buf_off_tiles[h->cur], h->buf_off_groups[h->cur], q, new_k, new_v, kv_cache, page_table,
+                                      cu_q_lens, kv_lens, out);
     a.group_counters = h->policy.fused_combine ? h->d_group_counters : nullptr;
     a.num_row_items = (int32_t)h->plan.rows.size();
     a.num_tile_items = (int32_t)h->plan.tiles.size();
@@ -594,7 +599,7 @@ rpa_status_t rpa_forward(rpa_handle_t* h, const void* q, const void* new_k, cons
     RPA_CUDA(h, cudaStreamWaitEvent(s, h->ev_copied[h->cur], 0));  // the plan's lists have landed
     if (h->validate) {
         a.validated = 1;
-        RPA_CUDA(h, launch_validate_kernel(a, num_seqs, reinterpret_cast<const int32_t*>(lists + h->off_kvlens), s));
+        RPA_CUDA(h, launch_validate_kernel(a, num_seqs, reinterpret_cast<const int32_t*>(lists + h->buf_off_kvlens[h->cur]), s));
     }
     const bool single_tile = tile1_kernel_supported(h->cfg.head_dim, h->cfg.num_q_heads / h->cfg.num_kv_heads);
     const bool side_by_side = a.num_row_items > 0 && a.num_tile_items > 0 && !(h->ablation & kAblateOverlap);
@@ -604,8 +609,8 @@ rpa_status_t rpa_forward(rpa_handle_t* h, const void* q, const void* new_k, cons
         RPA_CUDA(h, cudaEventRecord(h->ev_fork, s));
         RPA_CUDA(h, cudaStreamWaitEvent(h->aux_stream, h->ev_fork, 0));
         timing_mark(h, 1, h->aux_stream);
-        RPA_CUDA(h, single_tile ? launch_tile1_kernel(a, h->plan.info.num_tokens, h->aux_stream)
-                                : launch_tile_kernel(a, h->plan.info.num_tokens, h->aux_stream));
+        RPA_CUDA(h, single_tile ? launch_tile1_kernel(a, h->plan.info.num_tokens, &h->tile_maps, h->aux_stream)
+                                : launch_tile_kernel(a, h->plan.info.num_tokens, &h->tile_maps, h->aux_stream));
         timing_mark(h, 1, h->aux_stream);
         RPA_CUDA(h, cudaEventRecord(h->ev_join, h->aux_stream));
         timing_mark(h, 0, s);
@@ -621,8 +626,8 @@ rpa_status_t rpa_forward(rpa_handle_t* h, const void* q, const void* new_k, cons
         if (a.num_tile_items > 0) {
             a.num_tile_ctas = h->num_sms;  // one after the other: the whole device each, one persistent CTA per SM
             timing_mark(h, 1, s);
-            RPA_CUDA(h, single_tile ? launch_tile1_kernel(a, h->plan.info.num_tokens, s)
-                                    : launch_tile_kernel(a, h->plan.info.num_tokens, s));
+            RPA_CUDA(h, single_tile ? launch_tile1_kernel(a, h->plan.info.num_tokens, &h->tile_maps, s)
+                                    : launch_tile_kernel(a, h->plan.info.num_tokens, &h->tile_maps, s));
             timing_mark(h, 1, s);
         }
     }
@@ -684,15 +689,15 @@ rpa_status_t rpa_forward_host_submit(rpa_handle_t* h, const void* q_host, const 
         RPA_CUDA(h, cudaMemcpyAsync(d + h->hs_v, new_v_host, T * k_row, cudaMemcpyHostToDevice, h->h2d_stream));
         RPA_CUDA(h, cudaMemcpyAsync(d + h->hs_pt, page_table_host, (size_t)num_seqs * c.max_pages_per_seq * 4,
                                     cudaMemcpyHostToDevice, h->h2d_stream));
-        RPA_CUDA(h, cudaMemcpyAsync(d + h->hs_cu, cu_q_lens_host, ((size_t)num_seqs + 1) * 4, cudaMemcpyHostToDevice, h->h2d_stream));
-        RPA_CUDA(h, cudaMemcpyAsync(d + h->hs_kl, kv_lens_host, (size_t)num_seqs * 4, cudaMemcpyHostToDevice, h->h2d_stream));
+        // (the lengths travel with the plan's lists: one copy less each)
     }
     RPA_CUDA(h, cudaEventRecord(h->ev_in[slot], h->h2d_stream));
     RPA_CUDA(h, cudaStreamWaitEvent(s, h->ev_in[slot], 0));
     if (!empty) {
+        const uint8_t* lists = h->d_lists[h->cur];
         st = rpa_forward(h, d + h->hs_q, d + h->hs_k, d + h->hs_v, kv_cache, reinterpret_cast<const int32_t*>(d + h->hs_pt),
-                         reinterpret_cast<const int32_t*>(d + h->hs_cu), reinterpret_cast<const int32_t*>(d + h->hs_kl),
-                         num_seqs, d + h->hs_out, stream);
+                         reinterpret_cast<const int32_t*>(lists + h->buf_off_cu[h->cur]),
+                         reinterpret_cast<const int32_t*>(lists + h->buf_off_kvlens[h->cur]), num_seqs, d + h->hs_out, stream);
         if (st != RPA_OK) return st;
     }
     RPA_CUDA(h, cudaEventRecord(h->ev_ran[slot], s));

@@ -98,17 +98,33 @@ int row_kernel_fp8_narrow_ctas_per_sm(int head_dim);  // the 8-row instantiation
 cudaError_t row_kernel_fp8_prepare(int head_dim, int group);
 cudaError_t launch_row_kernel_fp8(const KernelArgs& a, cudaStream_t stream);
 
+// The tensor maps of a tile-kernel launch, kept from launch to launch: encoding the five maps costs
+// several microseconds of host time, and a serving loop passes the same tensors step after step.  An
+// entry is reused when every tensor address and extent it was built from matches (a few entries, so
+// that alternating staging buffers all hit); null: encode afresh.
+struct TileMapCache {
+    static constexpr int kEntries = 4;
+    struct Entry {
+        bool valid = false;
+        const void *q = nullptr, *out = nullptr, *new_k = nullptr, *new_v = nullptr, *kv_cache = nullptr;
+        int64_t token_rows = 0;
+        int32_t h_q = 0, h_kv = 0, head_dim = 0, page_size = 0, num_pages = 0, kv_fp8 = 0, block_n = 0, q_tile_tokens = 0;
+        alignas(64) unsigned char maps[5 * 128];  // five CUtensorMap objects (128 bytes each)
+    } entries[kEntries];
+    int next = 0;
+};
+
 bool tile_kernel_supported(int head_dim, int group);       // d_k = 256 does not fit its TMEM budget
 int tile_kernel_tokens(int group);                         // new tokens one tile item covers
 bool tile_kernel_fp8_supported(int head_dim, int group);   // the same kernel on an FP8 E4M3 cache
 cudaError_t tile_kernel_prepare(int head_dim, int group, bool fp8);  // opts in to its dynamic shared memory
 // token_rows: rows of q / new_k / new_v the call may touch (tensor-map extent; rows past it read as zero)
-cudaError_t launch_tile_kernel(const KernelArgs& a, int64_t token_rows, cudaStream_t stream);
+cudaError_t launch_tile_kernel(const KernelArgs& a, int64_t token_rows, TileMapCache* cache, cudaStream_t stream);
 
 // single-tile variant with double-buffered scores (rpa_tile1_kernel.cu): d_k = 256
 bool tile1_kernel_supported(int head_dim, int group);
 cudaError_t tile1_kernel_prepare(int head_dim, int group);
-cudaError_t launch_tile1_kernel(const KernelArgs& a, int64_t token_rows, cudaStream_t stream);
+cudaError_t launch_tile1_kernel(const KernelArgs& a, int64_t token_rows, TileMapCache* cache, cudaStream_t stream);
 
 // Checks the device copies of the lengths against the plan and every page id a sequence maps
 // against the pool size; a violation sets bit 29 of the status word (low bits: the sequence).

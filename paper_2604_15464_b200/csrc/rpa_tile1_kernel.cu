@@ -570,9 +570,9 @@ rpa_tile1_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
 }
 
 template <int D, int G>
-cudaError_t launch_tile1(const KernelArgs& a, int64_t token_rows, cudaStream_t stream) {
+cudaError_t launch_tile1(const KernelArgs& a, int64_t token_rows, TileMapCache* cache, cudaStream_t stream) {
     TileMaps maps;
-    if (!build_tile_maps(a, token_rows, D, G, 128 / G, Tile1Cfg<D>::BN, &maps)) return cudaErrorInvalidValue;
+    if (!cached_tile_maps(cache, a, token_rows, D, G, 128 / G, Tile1Cfg<D>::BN, &maps)) return cudaErrorInvalidValue;
     const int grid = a.dev_counts ? a.num_tile_ctas : a.num_tile_ctas > 0 && a.num_tile_ctas < a.num_tile_items ? a.num_tile_ctas : a.num_tile_items;
     if (a.kv_fp8) {  // the quantising pass first: cache update of the items' own tokens, bf16 copies of their codes
         if (cudaError_t e = launch_quantise_new<D>(a, stream); e != cudaSuccess) return e;
@@ -614,9 +614,9 @@ cudaError_t tile1_kernel_prepare(int head_dim, int group) {
     return cudaErrorInvalidValue;
 }
 
-cudaError_t launch_tile1_kernel(const KernelArgs& a, int64_t token_rows, cudaStream_t stream) {
+cudaError_t launch_tile1_kernel(const KernelArgs& a, int64_t token_rows, TileMapCache* cache, cudaStream_t stream) {
     if (a.num_tile_items <= 0 && !a.dev_counts) return cudaSuccess;
-    RPA_TILE1_DISPATCH(a.head_dim, a.h_q / a.h_kv, launch_tile1, a, token_rows, stream);
+    RPA_TILE1_DISPATCH(a.head_dim, a.h_q / a.h_kv, launch_tile1, a, token_rows, cache, stream);
     return cudaErrorInvalidValue;
 }
 

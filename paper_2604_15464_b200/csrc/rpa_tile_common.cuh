@@ -2,6 +2,7 @@
 #pragma once
 #include <cuda.h>
 #include <cuda_runtime.h>
+#include <string.h>
 
 #include "rpa_fp8.cuh"
 #include "rpa_kernels.h"
@@ -296,6 +297,34 @@ inline bool build_tile_maps(const KernelArgs& a, int64_t token_rows, int D, int 
         const uint32_t box[4] = {64, 1, (uint32_t)page_box_rows(a.page_size, block_n), 1};
         if (!make_map(&maps->cache, a.kv_cache, 4, dims, str, box)) return false;
     }
+    return true;
+}
+
+// The same through a cache (see TileMapCache): returns the launch's maps, encoding them only when
+// no entry was built from the same tensors.
+inline bool cached_tile_maps(TileMapCache* cache, const KernelArgs& a, int64_t token_rows, int D, int G, int q_tile_tokens,
+                             int block_n, TileMaps* maps) {
+    static_assert(sizeof(TileMaps) == 5 * 128, "five tensor maps");
+    if (!cache) return build_tile_maps(a, token_rows, D, G, q_tile_tokens, block_n, maps);
+    const void* nk = a.kv_fp8 ? (const void*)a.new_k_codes : (const void*)a.new_k;
+    const void* nv = a.kv_fp8 ? (const void*)a.new_v_codes : (const void*)a.new_v;
+    for (auto& e : cache->entries) {
+        if (e.valid && e.q == a.q && e.out == a.out && e.new_k == nk && e.new_v == nv && e.kv_cache == a.kv_cache &&
+            e.token_rows == token_rows && e.h_q == a.h_q && e.h_kv == a.h_kv && e.head_dim == D && e.page_size == a.page_size &&
+            e.num_pages == a.num_pages && e.kv_fp8 == a.kv_fp8 && e.block_n == block_n && e.q_tile_tokens == q_tile_tokens) {
+            memcpy(maps, e.maps, sizeof(TileMaps));
+            return true;
+        }
+    }
+    if (!build_tile_maps(a, token_rows, D, G, q_tile_tokens, block_n, maps)) return false;
+    auto& e = cache->entries[cache->next];
+    cache->next = (cache->next + 1) % TileMapCache::kEntries;
+    e.valid = true;
+    e.q = a.q, e.out = a.out, e.new_k = nk, e.new_v = nv, e.kv_cache = a.kv_cache;
+    e.token_rows = token_rows;
+    e.h_q = a.h_q, e.h_kv = a.h_kv, e.head_dim = D, e.page_size = a.page_size, e.num_pages = a.num_pages, e.kv_fp8 = a.kv_fp8;
+    e.block_n = block_n, e.q_tile_tokens = q_tile_tokens;
+    memcpy(e.maps, maps, sizeof(TileMaps));
     return true;
 }
 

@@ -785,9 +785,9 @@ rpa_tile_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
 // ---- host side -------------------------------------------------------------------------------
 
 template <int D, int G, bool FP8>
-cudaError_t launch_tile(const KernelArgs& a, int64_t token_rows, cudaStream_t stream) {
+cudaError_t launch_tile(const KernelArgs& a, int64_t token_rows, TileMapCache* cache, cudaStream_t stream) {
     TileMaps maps;
-    if (!build_tile_maps(a, token_rows, D, G, 128 / G, kBlockN, &maps)) return cudaErrorInvalidValue;
+    if (!cached_tile_maps(cache, a, token_rows, D, G, 128 / G, kBlockN, &maps)) return cudaErrorInvalidValue;
     if (FP8) {
         if (cudaError_t e = launch_quantise_new<D>(a, stream); e != cudaSuccess) return e;
     }
@@ -866,9 +866,9 @@ cudaError_t tile_kernel_prepare(int head_dim, int group, bool fp8) {
     return cudaErrorInvalidValue;
 }
 
-cudaError_t launch_tile_kernel(const KernelArgs& a, int64_t token_rows, cudaStream_t stream) {
+cudaError_t launch_tile_kernel(const KernelArgs& a, int64_t token_rows, TileMapCache* cache, cudaStream_t stream) {
     if (a.num_tile_items <= 0 && !a.dev_counts) return cudaSuccess;
-    RPA_TILE_DISPATCH(a.head_dim, a.h_q / a.h_kv, a.kv_fp8 != 0, launch_tile, a, token_rows, stream);
+    RPA_TILE_DISPATCH(a.head_dim, a.h_q / a.h_kv, a.kv_fp8 != 0, launch_tile, a, token_rows, cache, stream);
     return cudaErrorInvalidValue;
 }
 
