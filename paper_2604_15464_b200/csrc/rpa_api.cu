@@ -414,21 +414,40 @@ static rpa_status_t forward_device_planned(rpa_handle* h, const void* q, const v
     const bool capturing = stream_is_capturing(s);
     if (!capturing && h->dev_planned_pending[b]) RPA_CUDA(h, cudaStreamWaitEvent(s, h->ev_dev_planned[b], 0));  // the plan may come from another stream
     const bool tiles = h->policy.tile_min_q > 0;
-    if (tiles) {
-        RPA_CUDA(h, cudaEventRecord(h->ev_fork, s));
-        RPA_CUDA(h, cudaStreamWaitEvent(h->aux_stream, h->ev_fork, 0));
-        const bool single_tile = tile1_kernel_supported(c.head_dim, c.num_q_heads / c.num_kv_heads);
-        timing_mark(h, 1, h->aux_stream);
-        RPA_CUDA(h, single_tile ? launch_tile1_kernel(a, c.max_num_tokens, &h->tile_maps, h->aux_stream)
-                                : launch_tile_kernel(a, c.max_num_tokens, &h->tile_maps, h->aux_stream));
-        timing_mark(h, 1, h->aux_stream);
-        RPA_CUDA(h, cudaEventRecord(h->ev_join, h->aux_stream));
-    }
+    const bool single_tile = tile1_kernel_supported(c.head_dim, c.num_q_heads / c.num_kv_heads);
     // eight waves of resident CTAs: short lists get one item per CTA (placed dynamically by the
     // hardware, as with a host-made plan), long ones are strided
     const int grid = (int)std::min<int64_t>(h->policy.max_row_items, (int64_t)8 * h->policy.num_slots);
-    timing_mark(h, 0, s);
-    if (fp8) {
+    if (!fp8) {
+        // One stream, two kernels as a programmatic pair.  The tile kernel goes first and gets its SMs
+        // first (a CTA of it needs an SM to itself even to find that the list holds nothing for it);
+        // its CTAs signal at their start, and the row kernel's CTAs follow them onto the device without
+        // waiting for the tile kernel to end.  A decode step thus pays for a grid of CTAs that leave at
+        // once, not for a kernel that can only start as the row kernel drains.  (Events recorded
+        // between the two launches, when per-kernel timing is on, serialise the pair.)
+        if (tiles) {
+            a.pdl_primary = 1;
+            timing_mark(h, 1, s);
+            RPA_CUDA(h, single_tile ? launch_tile1_kernel(a, c.max_num_tokens, &h->tile_maps, s)
+                                    : launch_tile_kernel(a, c.max_num_tokens, &h->tile_maps, s));
+            timing_mark(h, 1, s);
+            a.pdl_primary = 0;
+            a.pdl_secondary = 1;
+        }
+        timing_mark(h, 0, s);
+        RPA_CUDA(h, launch_row_kernel_strided(a, grid, s));
+        timing_mark(h, 0, s);
+    } else {
+        if (tiles) {
+            RPA_CUDA(h, cudaEventRecord(h->ev_fork, s));
+            RPA_CUDA(h, cudaStreamWaitEvent(h->aux_stream, h->ev_fork, 0));
+            timing_mark(h, 1, h->aux_stream);
+            RPA_CUDA(h, single_tile ? launch_tile1_kernel(a, c.max_num_tokens, &h->tile_maps, h->aux_stream)
+                                    : launch_tile_kernel(a, c.max_num_tokens, &h->tile_maps, h->aux_stream));
+            timing_mark(h, 1, h->aux_stream);
+            RPA_CUDA(h, cudaEventRecord(h->ev_join, h->aux_stream));
+        }
+        timing_mark(h, 0, s);
         // Two instantiations, of which the list needs one (known on the device only): side by side, so
         // that the idle one's CTAs leave while the other one already works.
         const bool both = c.num_q_heads / c.num_kv_heads <= 8;
@@ -442,11 +461,9 @@ static rpa_status_t forward_device_planned(rpa_handle* h, const void* q, const v
         } else {
             RPA_CUDA(h, launch_row_kernel_fp8_strided(a, grid, false, s));
         }
-    } else {
-        RPA_CUDA(h, launch_row_kernel_strided(a, grid, s));
+        timing_mark(h, 0, s);
+        if (tiles) RPA_CUDA(h, cudaStreamWaitEvent(s, h->ev_join, 0));
     }
-    timing_mark(h, 0, s);
-    if (tiles) RPA_CUDA(h, cudaStreamWaitEvent(s, h->ev_join, 0));
     if (!capturing) {
         RPA_CUDA(h, cudaEventRecord(h->ev_dev_consumed[b], s));
         h->dev_consumed_pending[b] = true;

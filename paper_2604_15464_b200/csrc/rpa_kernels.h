@@ -29,7 +29,7 @@ struct KernelArgs {
     float* partial_o;   // [partials][16][d] unnormalised accumulators
     float* partial_ml;  // [partials][16][2] running max (log2 domain) and sum
     int32_t* group_counters;  // one arrival ticket per combine group (zero between calls); null: separate combine kernel
-    int32_t* tile_counters;   // [0] next tile item to draw, [1] CTAs that have left; both zero between launches
+    int32_t* tile_counters;   // [0] next tile item to draw, [1] tile CTAs that have left, [2] CTAs of a dependent row kernel that have finished; all zero between launches
     uint32_t* status;   // device status word
     int32_t num_row_items;
     int32_t num_tile_items;
@@ -53,6 +53,13 @@ struct KernelArgs {
     // Lists planned on the device: the counts live in device memory (written by the plan kernel of the
     // same step) and take the place of num_row_items, num_tile_items, num_groups and num_tile_ctas.
     const int32_t* dev_counts;  // null: the counts above hold
+    // Device-planned steps on a bf16 cache run the tile kernel and the row kernel on ONE stream as a
+    // programmatic pair: the tile kernel's CTAs signal at their start (pdl_primary), so the row kernel's
+    // CTAs follow them onto the SMs at once instead of waiting for the tile kernel to end, and the
+    // row kernel's CTAs wait for the tile kernel's completion only when they leave (pdl_secondary),
+    // which keeps the stream's order towards whatever comes next.
+    int32_t pdl_primary;
+    int32_t pdl_secondary;
 };
 
 enum { kDevCountRows = 0, kDevCountTiles = 1, kDevCountGroups = 2, kDevCountTileCtas = 3, kDevCountError = 4,
@@ -83,6 +90,7 @@ struct DevPlanArgs {
 };
 cudaError_t launch_plan_kernel(const DevPlanArgs& p, cudaStream_t stream);
 // the row kernel for device-planned lists: a fixed grid whose CTAs stride over the item list
+// (a.pdl_secondary: launched as the programmatic dependent of the kernel before it on `stream`)
 cudaError_t launch_row_kernel_strided(const KernelArgs& a, int grid, cudaStream_t stream);
 // narrow: the 8-row instantiation (a no-op for more than 8 grouped heads); a device-planned step launches both
 cudaError_t launch_row_kernel_fp8_strided(const KernelArgs& a, int grid, bool narrow, cudaStream_t stream);

@@ -355,7 +355,10 @@ __global__ void __launch_bounds__(RowCfg<D>::NW * 32, RowCfg<D>::CTAS_PER_SM) rp
 template <int D, int G>
 __global__ void __launch_bounds__(RowCfg<D>::NW * 32, RowCfg<D>::CTAS_PER_SM) rpa_row_kernel_strided(const KernelArgs a) {
     extern __shared__ __align__(128) uint8_t smem[];
-    if (*reinterpret_cast<volatile uint32_t*>(a.status) & kStatusBadInput) return;  // the planner rejected the lengths
+    if (*reinterpret_cast<volatile uint32_t*>(a.status) & kStatusBadInput) {  // the planner rejected the lengths
+        if (a.pdl_secondary && threadIdx.x == 0) pdl_wait();  // (every CTA comes this way: nothing to make room for)
+        return;
+    }
     const int n = a.dev_counts[kDevCountRows];
     // the list is sorted longest first: dealing it back and forth (CTA b takes b, 2G-1-b, 2G+b, ...)
     // pairs the longest items of one pass with the shortest of the next
@@ -365,6 +368,16 @@ __global__ void __launch_bounds__(RowCfg<D>::NW * 32, RowCfg<D>::CTAS_PER_SM) rp
         if (i >= n) continue;
         row_item<D, G>(a, i, smem);
         __syncthreads();  // the next item reuses the shared memory
+    }
+    // Launched as the programmatic dependent of the tile kernel: this kernel must not be seen as
+    // complete before that one is (what follows on the stream relies on both).  The last CTA to
+    // finish waits for it; the others leave and make room for the CTAs still to come.
+    if (a.pdl_secondary && threadIdx.x == 0) {
+        __threadfence();
+        if (atomicAdd(a.tile_counters + 2, 1) == (int)gridDim.x - 1) {
+            a.tile_counters[2] = 0;  // zero again for the next launch
+            pdl_wait();
+        }
     }
 }
 
@@ -401,8 +414,21 @@ cudaError_t launch_row(const KernelArgs& a, cudaStream_t stream) {
 
 template <int D, int G>
 cudaError_t launch_row_strided(const KernelArgs& a, int grid, cudaStream_t stream) {
-    rpa_row_kernel_strided<D, G><<<grid, RowCfg<D>::NW * 32, RowCfg<D>::SMEM, stream>>>(a);
-    return cudaGetLastError();
+    if (!a.pdl_secondary) {
+        rpa_row_kernel_strided<D, G><<<grid, RowCfg<D>::NW * 32, RowCfg<D>::SMEM, stream>>>(a);
+        return cudaGetLastError();
+    }
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(RowCfg<D>::NW * 32);
+    cfg.dynamicSmemBytes = RowCfg<D>::SMEM;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr{};
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, rpa_row_kernel_strided<D, G>, a);
 }
 
 template <int D, int G>

@@ -88,6 +88,9 @@ rpa_tile_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
     volatile int* item_slots = reinterpret_cast<volatile int*>(smem + C::OFF_BAR + 256);
     auto bar = [&](int slot) { return bars + 8u * slot; };
 
+    // first of a programmatic pair: the kernel behind this one on the stream may start as soon as
+    // every CTA of this one has got its SM (or has left)
+    if (a.pdl_primary && threadIdx.x == 0) pdl_launch_dependents();
     if ((a.validated || a.dev_counts) && (*reinterpret_cast<volatile uint32_t*>(a.status) & kStatusBadInput)) return;  // inputs were rejected
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     if (a.dev_counts && (int)blockIdx.x >= a.dev_counts[kDevCountTileCtas]) {
