@@ -241,8 +241,8 @@ rpa_status_t rpa_plan_dump(const rpa_handle_t* h, int32_t* row_items, int32_t ro
 /*
  * Device-side planner: the same plan as rpa_plan, built by a kernel on `stream` from the DEVICE
  * copies of the lengths (cu_q_lens [n+1], kv_lens [n], the pointers rpa_forward gets), with no host
- * round trip: the remedy for the metadata work the paper leaves on the critical path (Section 6,
- * future work).  The following rpa_forward with the same num_seqs launches fixed grids that read
+ * round trip: the remedy for the metadata work the paper leaves on the critical path (Section 5,
+ * Discussion and Future Directions).  The following rpa_forward with the same num_seqs launches fixed grids that read
  * their item counts from device memory, so the pair may be captured in a CUDA graph and replayed
  * after the caller has changed the lengths, page table and inputs in place.  Differences from
  * rpa_plan: runs of short sequences are packed into shared tile items only in batches of up to 1024
@@ -250,7 +250,10 @@ rpa_status_t rpa_plan_dump(const rpa_handle_t* h, int32_t* row_items, int32_t ro
  * tensor maps cover that extent).  Invalid
  * lengths or a batch beyond the handle's capacities are found on the device: the step's kernels
  * then do nothing and rpa_poll_status reports RPA_ERR_INVALID_ARG (bit 29 of the word; bit 20:
- * bad lengths, bit 21: capacity).  The first call allocates the device lists and scratch - make it
+ * bad lengths, bit 21: capacity).  That word is STICKY: until rpa_poll_status has reported and cleared
+ * it, every later device-planned step (and every later validated host-planned step) also returns at
+ * once without writing `out` or the cache - a loop that replays a graph and polls only now and then
+ * drops steps in the meantime.  The first call allocates the device lists and scratch - make it
  * before capturing.  rpa_plan_info and rpa_plan_dump do not describe a device-made plan, and
  * rpa_set_validation has no effect on a device-planned step.
  * Streams: the handle keeps two sets of device lists.  Outside a capture, each rpa_plan_device
@@ -289,8 +292,14 @@ rpa_status_t rpa_poll_status(rpa_handle_t* h, void* stream, uint32_t* detail);
  * kernel that checks, for every sequence, that the device copy of kv_lens equals the planned one and
  * that every page id the sequence maps lies in [0, num_pages).  On a violation bit 29 of the status
  * word is set (low 20 bits: a sequence at fault), the attention kernels of that call return at once
- * without touching kv_cache or out, and rpa_poll_status reports RPA_ERR_INVALID_ARG.  Costs one extra
- * launch per call.
+ * without touching kv_cache or out, and rpa_poll_status reports RPA_ERR_INVALID_ARG.  The word stays
+ * set until it is polled, and while it is set every later validated call returns at once in the same
+ * way.  Costs one extra launch per call.
+ *
+ * Bounds-checked build: `librpa_b200_debug.so` (python -m paper_2604_15464_b200.build --debug) is the
+ * same library compiled with -DRPA_DEBUG.  Its kernels check every page id, token row and ring stage
+ * before the access; the first violation of a call sets bit 27 of the status word (bits 24..26: 1 page
+ * id, 2 token row, 3 stage index; low 24 bits: the offending value) and the access is skipped.
  */
 rpa_status_t rpa_set_validation(rpa_handle_t* h, int32_t enable);
 

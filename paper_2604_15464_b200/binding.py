@@ -151,8 +151,9 @@ def rpa_forward_static(config: RpaConfig, q, new_k, new_v, kv_cache, page_table,
 class Rpa:
     """One library handle.  ``device`` < 0 gives a planning-only handle that makes no CUDA call."""
 
-    def __init__(self, config: RpaConfig, device: int = 0):
-        self._lib = load_library()
+    def __init__(self, config: RpaConfig, device: int = 0, library_path: Optional[str] = None):
+        # library_path: another build of the same library (the bounds-checked one, say)
+        self._lib = load_library(library_path)
         self.config = config
         self.device = device
         self._h = ctypes.c_void_p()
@@ -167,9 +168,10 @@ class Rpa:
         cfg = RpaConfig(meta.num_q_heads, meta.num_kv_heads, meta.head_dim, meta.page_size, meta.num_pages,
                         meta.max_pages_per_seq, max(meta.num_seqs, 1), max(meta.token_capacity, 1), meta.scale,
                         meta.causal, meta.kv_fp8, meta.k_scale, meta.v_scale)
+        library_path = over.pop("library_path", None)
         for k, v in over.items():
             setattr(cfg, k, v)
-        return cls(cfg, device)
+        return cls(cfg, device, library_path)
 
     def close(self) -> None:
         if getattr(self, "_h", None) and self._h.value:

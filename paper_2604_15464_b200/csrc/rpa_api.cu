@@ -2,6 +2,7 @@
 #include <cuda_runtime.h>
 #include <math.h>
 #include <stdio.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include <algorithm>
@@ -189,6 +190,30 @@ bool tile_path_available(const rpa_config_t& c) {
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+// RPA_LOG=1 in the environment (read once): every rpa_plan prints one line to stderr that says what
+// it made of the batch - its class, how the sequences were routed, the work lists, the split-KV
+// chunk, the SM split of a mixed batch, the algorithmic work.
+bool plan_log_enabled() {
+    static const bool on = [] {
+        const char* v = getenv("RPA_LOG");
+        return v && *v && strcmp(v, "0") != 0;
+    }();
+    return on;
+}
+
+void log_plan(const rpa_handle* h) {
+    static const char* const kCase[] = {"empty", "decode", "prefill", "mixed"};
+    const rpa_plan_info_t& i = h->plan.info;
+    fprintf(stderr,
+            "[rpa] plan: %s batch, %d seqs (%d decode, %d prefill), %d new tokens; row kernel %d items (largest %d rows, "
+            "split chunk %d tokens, %d combine groups, %d partials), tile kernel %d items on %d CTAs; %d launches, %.3f GB, "
+            "%.3f GFLOP (row %.3f GB, tile %.3f GFLOP)\n",
+            kCase[i.batch_case & 3], i.num_seqs, i.num_decode_seqs, i.num_prefill_seqs, i.num_tokens, i.num_row_items,
+            h->plan.row_rows_max, i.kv_chunk_tokens, i.num_combine_groups, h->plan.num_partials, i.num_tile_items,
+            h->plan.tile_ctas > 0 ? h->plan.tile_ctas : (i.num_tile_items > 0 ? std::min(i.num_tile_items, h->num_sms) : 0),
+            i.gpu_launches, i.algorithmic_bytes / 1e9, i.algorithmic_flops / 1e9, i.row_bytes / 1e9, i.tile_flops / 1e9);
+}
+
 // Events recorded outside a capture cannot be waited for inside one (and the other way round): while
 // a stream is being captured into a graph, the capture's own order stands in for the handle's events.
 bool stream_is_capturing(cudaStream_t s) {
@@ -309,6 +334,7 @@ rpa_status_t rpa_plan(rpa_handle_t* h, const int32_t* cu_q_lens_host, const int3
     h->device_planned = false;
     rpa_status_t st = build_plan(h->cfg, h->policy, cu_q_lens_host, kv_lens_host, num_seqs, h->plan);
     if (st != RPA_OK) return st;
+    if (plan_log_enabled()) log_plan(h);
     if (!h->plan_only) {
         st = ensure_device(h);
         if (st != RPA_OK) return st;
@@ -388,6 +414,7 @@ static KernelArgs common_kernel_args(const rpa_handle* h, uint8_t* lists, size_t
     a.inv_k_scale = fp8 ? 1.0f / c.k_scale : 1.f;
     a.inv_v_scale = fp8 ? 1.0f / c.v_scale : 1.f;
     a.ablation = h->ablation;
+    a.token_cap = c.max_num_tokens;
     return a;
 }
 

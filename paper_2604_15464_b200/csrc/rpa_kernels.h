@@ -60,6 +60,7 @@ struct KernelArgs {
     // which keeps the stream's order towards whatever comes next.
     int32_t pdl_primary;
     int32_t pdl_secondary;
+    int32_t token_cap;  // rows of q / new_k / new_v / out the call may touch (checked by the RPA_DEBUG build)
 };
 
 enum { kDevCountRows = 0, kDevCountTiles = 1, kDevCountGroups = 2, kDevCountTileCtas = 3, kDevCountError = 4,
@@ -138,6 +139,61 @@ cudaError_t launch_tile1_kernel(const KernelArgs& a, int64_t token_rows, TileMap
 // against the pool size; a violation sets bit 29 of the status word (low bits: the sequence).
 cudaError_t launch_validate_kernel(const KernelArgs& a, int32_t num_seqs, const int32_t* plan_kv_lens, cudaStream_t stream);
 constexpr uint32_t kStatusBadInput = 1u << 29;
+
+// The bounds-checked build (-DRPA_DEBUG: a library of its own, see build.py) checks every page id
+// the kernels take from the page table, the token rows of every work item and the ring-stage
+// addresses they form, BEFORE the access.  The first violation of a call is recorded in the status
+// word - bit 27, the kind in bits 24..26, the offending value (page id, token row, stage index) in
+// the low 24 bits - and the access is skipped (a read goes to page 0 instead, a write is dropped, an
+// item with bad rows is not run): the stand-in for a memory checker where none may be run.  Never
+// traps.  In the normal build the helpers compile to nothing.
+constexpr uint32_t kStatusDebug = 1u << 27;
+enum { kDebugPageId = 1, kDebugTokenRow = 2, kDebugStage = 3 };
+#if defined(__CUDACC__)
+__device__ __forceinline__ void debug_record(const KernelArgs& a, int kind, int value) {
+    atomicCAS(a.status, 0u, kStatusDebug | ((uint32_t)kind << 24) | ((uint32_t)value & 0xFFFFFFu));  // the first one stays
+}
+// page id for a read: the id itself, or page 0 after recording an id outside the pool
+__device__ __forceinline__ int debug_read_page(const KernelArgs& a, int page) {
+#ifdef RPA_DEBUG
+    if ((unsigned)page >= (unsigned)a.num_pages) {
+        debug_record(a, kDebugPageId, page);
+        return 0;
+    }
+#endif
+    return page;
+}
+// may this page id be written through?
+__device__ __forceinline__ bool debug_write_page_ok(const KernelArgs& a, int page) {
+#ifdef RPA_DEBUG
+    if ((unsigned)page >= (unsigned)a.num_pages) {
+        debug_record(a, kDebugPageId, page);
+        return false;
+    }
+#endif
+    return true;
+}
+// do token rows [row0, row0 + n) lie inside the tensors?
+__device__ __forceinline__ bool debug_rows_ok(const KernelArgs& a, long long row0, int n) {
+#ifdef RPA_DEBUG
+    if (row0 < 0 || n < 0 || row0 + n > a.token_cap) {
+        debug_record(a, kDebugTokenRow, (int)(row0 + n));
+        return false;
+    }
+#endif
+    return true;
+}
+// is ring stage `index` one of the `stages` the ring has?
+__device__ __forceinline__ bool debug_stage_ok(const KernelArgs& a, int index, int stages) {
+#ifdef RPA_DEBUG
+    if ((unsigned)index >= (unsigned)stages) {
+        debug_record(a, kDebugStage, index);
+        return false;
+    }
+#endif
+    return true;
+}
+#endif
 
 // Launches one warp whose bounded wait must give up (nothing arrives): sets the status word.
 cudaError_t launch_wait_selftest(uint32_t* status, cudaStream_t stream);

@@ -123,7 +123,7 @@ rpa_status_t build_plan(const rpa_config_t& cfg, const PlanPolicy& policy, const
     const int64_t T = cu_q_lens[num_seqs];
     if (T > cfg.max_num_tokens) return RPA_ERR_CAPACITY;
 
-    // split-KV chunk: no item longer than a quarter of a slot's average share, never below 256
+    // split-KV chunk: no item longer than half (1 / kChunkDivisor) of a slot's average share, never below 256
     const int num_slots = policy.num_slots_narrow > 0 && row_rows <= 8 ? policy.num_slots_narrow : policy.num_slots;
     int64_t chunk = policy.kv_chunk_override;
     if (chunk <= 0) {

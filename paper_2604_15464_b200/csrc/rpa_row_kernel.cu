@@ -71,6 +71,7 @@ __device__ __forceinline__ void row_item(const KernelArgs& a, int item_index, ui
     const int ps = a.page_size;
     const int64_t slot_elems = (int64_t)2 * a.h_kv * D;  // elements between consecutive cache slots
     const int64_t tok0 = (int64_t)cu + it.q_tok0;
+    if (!debug_rows_ok(a, tok0, it.n_tok)) return;  // (bounds-checked build only)
 
     // ---- this warp's share of the KV tiles ----
     const int t_begin = it.kv_begin / kKvTile;
@@ -85,10 +86,11 @@ __device__ __forceinline__ void row_item(const KernelArgs& a, int item_index, ui
             const int pos0 = t * kKvTile;
             page_reg = (t < t_end && pos0 < c) ? pt_row[pos0 / ps] : 0;
         }
-        const int page = __shfl_sync(0xffffffffu, page_reg, kl & 31);
+        const int page = debug_read_page(a, __shfl_sync(0xffffffffu, page_reg, kl & 31));
         if (kl < n_my && !(a.ablation & kAblateLoads)) {
             const int pos0 = (t_begin + warp + kl * NW) * kKvTile;
             const uint32_t stage = ring + (kl % STAGES) * C::STAGE;
+            if (!debug_stage_ok(a, kl % STAGES, STAGES)) return;
             if (pos0 + kKvTile <= fast_end) {
                 const uint16_t* base = a.kv_cache + ((int64_t)page * ps + pos0 % ps) * slot_elems + (int64_t)2 * h * D;
 #pragma unroll
@@ -110,7 +112,7 @@ __device__ __forceinline__ void row_item(const KernelArgs& a, int item_index, ui
                     if (p >= it.kv_end) {
                         bytes = 0;  // zero-fill: masked scores, and finite V rows for the PV product
                     } else if (p < c) {
-                        const int pg = pt_row[p / ps];
+                        const int pg = debug_read_page(a, pt_row[p / ps]);
                         src = a.kv_cache + ((int64_t)pg * ps + p % ps) * slot_elems + (int64_t)2 * h * D + cc * 8;
                     } else {
                         src = (is_v ? a.new_v : a.new_k) + (((int64_t)cu + (p - c)) * a.h_kv + h) * D + ch * 8;
@@ -132,6 +134,7 @@ __device__ __forceinline__ void row_item(const KernelArgs& a, int item_index, ui
             const int j = idx / CPP, cc = idx % CPP;
             const int pos = c + it.q_tok0 + j;
             const int page = pt_row[pos / ps];
+            if (!debug_write_page_ok(a, page)) continue;
             uint16_t* dst = a.kv_cache + ((int64_t)page * ps + pos % ps) * slot_elems + (int64_t)2 * h * D + cc * 8;
             const uint16_t* src = (cc < CPR ? a.new_k : a.new_v) + ((tok0 + j) * a.h_kv + h) * D + (cc % CPR) * 8;
             *reinterpret_cast<uint4*>(dst) = ld_global_nc_v4(src);

@@ -93,6 +93,7 @@ __device__ __forceinline__ void row_item_fp8(const KernelArgs& a, int item_index
     const int ps = a.page_size;
     const int64_t slot_bytes = (int64_t)2 * a.h_kv * D;  // one byte per element
     const int64_t tok0 = (int64_t)cu + it.q_tok0;
+    if (!debug_rows_ok(a, tok0, it.n_tok)) return;  // (bounds-checked build only)
     uint8_t* cache8 = reinterpret_cast<uint8_t*>(a.kv_cache);
 
     // ---- this warp's share of the KV tiles ----
@@ -109,10 +110,11 @@ __device__ __forceinline__ void row_item_fp8(const KernelArgs& a, int item_index
             const int pos0 = t * kKvTile;
             page_reg = (t < t_end && pos0 < c) ? pt_row[pos0 / ps] : 0;
         }
-        const int page = __shfl_sync(0xffffffffu, page_reg, kl & 31);
+        const int page = debug_read_page(a, __shfl_sync(0xffffffffu, page_reg, kl & 31));
         if (kl < n_my && !(a.ablation & kAblateLoads)) {
             const int pos0 = (t_begin + warp + kl * NW) * kKvTile;
             const int stage_off = (kl % STAGES) * C::STAGE;
+            if (!debug_stage_ok(a, kl % STAGES, STAGES)) return;
             if (pos0 + kKvTile <= fast_end) {
                 const uint8_t* base = cache8 + ((int64_t)page * ps + pos0 % ps) * slot_bytes + (int64_t)2 * h * D;
 #pragma unroll
@@ -139,7 +141,7 @@ __device__ __forceinline__ void row_item_fp8(const KernelArgs& a, int item_index
                         const uint8_t* src = cache8;
                         uint32_t bytes = 0;  // past kv_end: zero-fill (masked scores, finite V rows)
                         if (p < c) {
-                            const int pg = pt_row[p / ps];
+                            const int pg = debug_read_page(a, pt_row[p / ps]);
                             src = cache8 + ((int64_t)pg * ps + p % ps) * slot_bytes + (int64_t)2 * h * D + cc * 16;
                             bytes = 16;
                         }
@@ -163,6 +165,7 @@ __device__ __forceinline__ void row_item_fp8(const KernelArgs& a, int item_index
             const int ch = cc - (is_v ? CPR : 0);
             const int pos = c + it.q_tok0 + j;
             const int page = pt_row[pos / ps];
+            if (!debug_write_page_ok(a, page)) continue;
             uint8_t* dst = cache8 + ((int64_t)page * ps + pos % ps) * slot_bytes + (int64_t)2 * h * D + cc * 16;
             const uint16_t* src = (is_v ? a.new_v : a.new_k) + ((tok0 + j) * a.h_kv + h) * D + ch * 16;
             *reinterpret_cast<uint4*>(dst) = quantise16(src, is_v ? a.inv_v_scale : a.inv_k_scale);

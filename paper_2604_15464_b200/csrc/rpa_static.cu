@@ -148,6 +148,7 @@ extern "C" rpa_status_t rpa_forward_static(const rpa_config_t* cfg, const void* 
     a.causal = c.causal ? 1 : 0;
     a.scale_log2 = c.sm_scale * 1.4426950408889634f;
     a.out_scale = 1.f;
+    a.token_cap = c.max_num_tokens;
     e = launch_row_kernel(a, s);
     if (e == cudaSuccess) e = launch_combine_kernel(a, s);
     return e == cudaSuccess ? RPA_OK : RPA_ERR_CUDA;

@@ -151,6 +151,7 @@ rpa_tile1_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
         tc_fence_after();
         if (slot[RAW_ITEM] >= n_items) break;
         const TileCtx it = tile_ctx_from_raw(a, slot, BN);
+      if (!debug_rows_ok(a, (long long)it.cu + it.q_tok0, it.n_tok)) break;  // (bounds-checked build: every thread of the CTA takes this exit together)
         const int h = it.h, cu = it.cu, q_r = it.q_r, L = it.L, c = it.c;
         const int n_ctx_blocks = it.n_ctx_blocks, n_new_visible = it.n_new_visible, n_blocks = it.n_blocks;
         const int32_t* pt_row = it.pt_row;
@@ -187,7 +188,7 @@ rpa_tile1_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
                     const int pos = j * BN + lane * box_rows;
                     sub_valid = lane < sub_blocks && pos < c;
                     if (sub_valid) {
-                        page = pt_row[pos / ps];
+                        page = debug_read_page(a, pt_row[pos / ps]);
                         slot0 = pos % ps;
                     }
                     n_sub_valid = __popc(__ballot_sync(0xffffffffu, sub_valid));

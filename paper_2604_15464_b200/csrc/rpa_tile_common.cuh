@@ -150,6 +150,7 @@ __device__ __forceinline__ bool tile_update_cache(const KernelArgs& a, const Til
             pt_row += (int64_t)k * a.max_pages_per_seq;
         }
         const int page = act ? pt_row[pos / ps] : 0;
+        const bool store_ok = act && debug_write_page_ok(a, page);  // (always true outside the bounds-checked build)
         if (lane == 0) sm100::mbar_arrive_expect_tx(bar, (uint32_t)nt * 2 * ROW);
         __syncwarp();
         if (act) {
@@ -158,7 +159,7 @@ __device__ __forceinline__ bool tile_update_cache(const KernelArgs& a, const Til
             sm100::bulk_load(mine + ROW, a.new_v + src, ROW, bar);
         }
         if (!sm100::mbar_wait(bar, round & 1, abort_flag, status, 0x40 + w)) return false;
-        if (act) {
+        if (store_ok) {
             sm100::bulk_store(a.kv_cache + ((int64_t)page * ps + pos % ps) * slot_elems + (int64_t)2 * it.h * D, mine, 2 * ROW);
             sm100::bulk_commit();
             sm100::bulk_wait_read();  // the staging area is free again
@@ -205,8 +206,9 @@ __global__ void __launch_bounds__(128) rpa_quantise_new_kernel(const KernelArgs 
         const uint4 codes = quantise16((kv ? a.new_v : a.new_k) + src, kv ? a.inv_v_scale : a.inv_k_scale);
         if (!(a.ablation & kAblateUpdate)) {
             const int page = pt[pos / a.page_size];
-            *reinterpret_cast<uint4*>(cache + ((int64_t)page * a.page_size + pos % a.page_size) * slot_bytes +
-                                      (int64_t)(2 * it.kv_head + kv) * D + piece * 16) = codes;
+            if (debug_write_page_ok(a, page))
+                *reinterpret_cast<uint4*>(cache + ((int64_t)page * a.page_size + pos % a.page_size) * slot_bytes +
+                                          (int64_t)(2 * it.kv_head + kv) * D + piece * 16) = codes;
         }
         uint4 lo, hi;
         lo.x = e4m3x2_to_bf16x2(codes.x & 0xffffu);

@@ -161,6 +161,7 @@ rpa_tile_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
       tc_fence_after();
       if (slot[RAW_ITEM] >= n_items) break;
       const TileCtx it = tile_ctx_from_raw(a, slot, kBlockN);
+      if (!debug_rows_ok(a, (long long)it.cu + it.q_tok0, it.n_tok)) break;  // (bounds-checked build: every thread of the CTA takes this exit together)
       const int h = it.h, cu = it.cu, q_r = it.q_r, c = it.c;
       const int n_ctx_blocks = it.n_ctx_blocks, n_new_visible = it.n_new_visible, n_blocks = it.n_blocks;
       const int32_t* pt_row = it.pt_row;
@@ -206,7 +207,7 @@ rpa_tile_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
                 const int pos = j * kBlockN + lane * box_rows;
                 sub_valid = lane < sub_blocks && pos < c;
                 if (sub_valid) {
-                    page = pt_row[pos / ps];
+                    page = debug_read_page(a, pt_row[pos / ps]);
                     slot0 = pos % ps;
                 }
                 n_sub_valid = __popc(__ballot_sync(0xffffffffu, sub_valid));
@@ -216,6 +217,7 @@ rpa_tile_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
 #pragma unroll
             for (int kv = 0; kv < 2; ++kv) {  // 0: K stage, 1: V stage
                 const int st = j & 1;
+                if (!debug_stage_ok(a, st, C::KS)) break;
                 const int full = (kv ? BAR_VFULL : BAR_KFULL) + st, empty = (kv ? BAR_VEMPTY : BAR_KEMPTY) + st;
                 if (j >= 2) ok = ok && mbar_wait(bar(empty), ((j >> 1) - 1) & 1, abort_flag, a.status, 0x10 + kv);
                 ok = __all_sync(0xffffffffu, ok);
@@ -540,6 +542,7 @@ rpa_tile_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
         const volatile int* slot = item_slots + (iter & 1) * RAW_INTS;
         if (slot[RAW_ITEM] >= n_items) break;
         const TileCtx it = tile_ctx_from_raw(a, slot, kBlockN);
+      if (!debug_rows_ok(a, (long long)it.cu + it.q_tok0, it.n_tok)) break;  // (bounds-checked build: every thread of the CTA takes this exit together)
         const int h = it.h, cu = it.cu, q_r = it.q_r, L = it.L, c = it.c;
         const int n_ctx_blocks = it.n_ctx_blocks, n_new_visible = it.n_new_visible, n_blocks = it.n_blocks;
         const uint32_t q_off = (iter & 1) ? C::OFF_K : C::OFF_QA;  // this item's query region (see the producer)

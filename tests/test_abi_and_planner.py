@@ -261,3 +261,27 @@ def test_fp8_lists_of_decode_sized_items_are_planned_for_more_resident_ctas():
     assert narrow[0] < wide[0] and narrow[1] > wide[1] and narrow[1] % 8 == 0
     two_tokens = chunk_and_items([2] * 40, [6001] * 40, True)   # 2 tokens x 4 heads = 8 rows: still narrow
     assert two_tokens == narrow
+
+
+def test_rpa_log_prints_one_plan_summary_per_call():
+    """RPA_LOG=1 in the environment: rpa_plan describes on stderr what it made of the batch."""
+    import subprocess
+    import sys
+
+    code = ("import sys; sys.path.insert(0, %r)\n"
+            "from paper_2604_15464_b200 import binding, build, workloads as wl\n"
+            "build.build()\n"
+            "for cfg in (2, 4):\n"
+            "    meta = wl.workload_meta(cfg)\n"
+            "    r = binding.Rpa.for_meta(meta, device=-1)\n"
+            "    r.rpa_plan(meta.cu_q_lens, meta.kv_lens)\n" % ROOT)
+    env = dict(os.environ, RPA_LOG="1")
+    res = subprocess.run([sys.executable, "-c", code], env=env, capture_output=True, text=True, timeout=600)
+    assert res.returncode == 0, res.stderr[-1500:]
+    lines = [l for l in res.stderr.splitlines() if l.startswith("[rpa] plan:")]
+    assert len(lines) == 2
+    assert "decode batch, 256 seqs (256 decode, 0 prefill), 256 new tokens" in lines[0] and "tile kernel 0 items" in lines[0]
+    assert "mixed batch, 200 seqs (192 decode, 8 prefill), 4288 new tokens" in lines[1]
+    quiet = subprocess.run([sys.executable, "-c", code], env={k: v for k, v in os.environ.items() if k != "RPA_LOG"},
+                           capture_output=True, text=True, timeout=600)
+    assert "[rpa] plan:" not in quiet.stderr

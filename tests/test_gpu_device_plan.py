@@ -203,3 +203,27 @@ def test_next_step_planned_on_a_side_stream_while_the_previous_one_runs():
         T = metas[k].num_tokens
         hz.compare_outputs(wl.bf16_bits(out)[:T], ref, metas[k].name)
         assert np.array_equal(wl.bf16_bits(batch.kv_cache), host["kv_cache"])
+
+
+def test_a_rejected_step_keeps_later_steps_from_running_until_the_status_is_polled():
+    """The status word set by a rejected device-planned step is sticky: every later step returns at once,
+    writing neither `out` nor the cache, until rpa_poll_status has reported (and cleared) it.  A loop that
+    replays a graph and polls rarely must know that it drops steps meanwhile."""
+    shape = dict(num_q_heads=32, num_kv_heads=8, head_dim=128, page_size=16)
+    meta = wl.build_meta("sticky", [1, 30, 2], [300, 130, 64], seed=9, **shape)
+    batch = wl.materialize(meta, _dev())
+    rapi = binding.Rpa.for_meta(meta)
+    out = torch.full(batch.q.shape, hz.SENTINEL, dtype=torch.int16, device=_dev()).view(torch.bfloat16)
+    before = wl.bf16_bits(batch.kv_cache).copy()
+    bad_kv = batch.kv_lens.clone()
+    bad_kv[1] = 3  # kv_len < q_len
+    rapi.rpa_plan_device(batch.cu_q_lens, bad_kv)
+    rapi.rpa_forward(batch.q, batch.new_k, batch.new_v, batch.kv_cache, batch.page_table, batch.cu_q_lens, bad_kv, out)
+    # a good step right behind it, no poll in between: skipped
+    rapi.rpa_plan_device(batch.cu_q_lens, batch.kv_lens)
+    rapi.rpa_forward(batch.q, batch.new_k, batch.new_v, batch.kv_cache, batch.page_table, batch.cu_q_lens, batch.kv_lens, out)
+    torch.cuda.synchronize()
+    assert np.all(wl.bf16_bits(out) == hz.SENTINEL) and np.array_equal(before, wl.bf16_bits(batch.kv_cache))
+    assert rapi.rpa_poll_status() & (1 << 29)
+    assert rapi.rpa_poll_status() == 0
+    hz.full_parity(batch, rapi=rapi, device_plan=True)  # after the poll the same step runs
