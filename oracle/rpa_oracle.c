@@ -35,6 +35,9 @@
  * every key and value, the batch's own new tokens included, back from the cache, i.e. in
  * quantised precision (Algorithm 1 composes its KV block in the cache's type and writes that same
  * block back).  The paper does not spell out the conversion; this is the reading taken.
+ * Section 3.8 gives Q a scalar scale of its own as well: with q_scale > 0 (FP8 cache only) every
+ * query element is taken in E4M3 precision too, as  e4m3(float(q) * (1.0f / q_scale)) * q_scale  --
+ * the same conversion as for K -- before the scores are formed; q_scale = 0 leaves Q in bf16.
  *
  * Layouts (row-major): q [T, h_q, d], new_k/new_v [T, h_kv, d],
  * kv_cache [num_pages, page_size, 2*h_kv, d], all bf16 bit patterns in
@@ -61,6 +64,7 @@ typedef struct {
     int32_t kv_fp8; /* 0: bf16 cache, 1: FP8 E4M3 cache with per-tensor scales */
     float k_scale;
     float v_scale;
+    float q_scale; /* > 0: Q is quantised to E4M3 with this per-tensor scale (FP8 cache only); 0: Q stays bf16 */
 } oracle_shape_t;
 
 static double bf16_to_double(uint16_t bits) {
@@ -124,6 +128,7 @@ int rpa_oracle_check(const oracle_shape_t *sh, const int32_t *page_table, const 
                      const int32_t *kv_lens, int num_seqs) {
     if (sh->num_kv_heads <= 0 || sh->num_q_heads % sh->num_kv_heads != 0) return -1;
     if (sh->kv_fp8 && !(sh->k_scale > 0.f && sh->v_scale > 0.f)) return -8;
+    if (!(sh->q_scale >= 0.f) || (sh->q_scale > 0.f && !sh->kv_fp8)) return -9;
     if (cu_q_lens[0] != 0) return -2;
     for (int r = 0; r < num_seqs; ++r) {
         int q_r = cu_q_lens[r + 1] - cu_q_lens[r];
@@ -188,6 +193,15 @@ static void attend_one(const oracle_shape_t *sh, const uint16_t *q, const uint16
     const uint16_t *q_row = q + (((int64_t)cu_q_lens[r] + i) * sh->num_q_heads + a) * d;
 
     const uint8_t *cache8 = (const uint8_t *)kv_cache;
+    /* the query row as the scores see it: bf16, or its E4M3 image under the per-tensor scale of Q */
+    double *q_val = (double *)malloc(sizeof(double) * (size_t)d);
+    for (int e = 0; e < d; ++e) {
+        q_val[e] = bf16_to_double(q_row[e]);
+        if (sh->q_scale > 0.f) {
+            const float inv_q = 1.0f / sh->q_scale;
+            q_val[e] = rpa_oracle_e4m3_to_double(rpa_oracle_float_to_e4m3((float)q_val[e] * inv_q)) * (double)sh->q_scale;
+        }
+    }
     double M = -INFINITY;
     for (int64_t t = 0; t <= hi; ++t) {
         const int64_t k_off = slot_offset(sh, page_table, r, t, 2 * h);
@@ -195,7 +209,7 @@ static void attend_one(const oracle_shape_t *sh, const uint16_t *q, const uint16
         for (int e = 0; e < d; ++e) {
             double k_val = sh->kv_fp8 ? rpa_oracle_e4m3_to_double(cache8[k_off + e]) * (double)sh->k_scale
                                       : bf16_to_double(kv_cache[k_off + e]);
-            dot += bf16_to_double(q_row[e]) * k_val;
+            dot += q_val[e] * k_val;
         }
         score[t] = sh->scale * dot;
         if (score[t] > M) M = score[t];
@@ -213,6 +227,7 @@ static void attend_one(const oracle_shape_t *sh, const uint16_t *q, const uint16
         }
     }
     for (int e = 0; e < d; ++e) out_row[e] /= Z;
+    free(q_val);
 }
 
 /*

@@ -45,6 +45,7 @@ class _Shape(ctypes.Structure):
         ("kv_fp8", ctypes.c_int32),
         ("k_scale", ctypes.c_float),
         ("v_scale", ctypes.c_float),
+        ("q_scale", ctypes.c_float),
     ]
 
 
@@ -61,11 +62,12 @@ class OracleShape:
     kv_fp8: bool = False  # FP8 E4M3 cache (uint8 codes) with per-tensor scales
     k_scale: float = 1.0
     v_scale: float = 1.0
+    q_scale: float = 0.0  # > 0: Q is taken in E4M3 precision with this per-tensor scale (FP8 cache only)
 
     def _c(self) -> _Shape:
         return _Shape(self.num_q_heads, self.num_kv_heads, self.head_dim, self.page_size, self.num_pages,
                       self.max_pages_per_seq, 1 if self.causal else 0, float(self.scale), 1 if self.kv_fp8 else 0,
-                      float(self.k_scale), float(self.v_scale))
+                      float(self.k_scale), float(self.v_scale), float(self.q_scale))
 
     @property
     def cache_dtype(self):

@@ -111,3 +111,76 @@ def test_fp8_forward_matches_dense_attention_on_dequantised_kv(case, causal):
             S = S.masked_fill((key > qpos)[None], float("-inf"))
         ref = torch.einsum("ait,tad->iad", torch.softmax(S, dim=-1), V).numpy()
         assert np.max(np.abs(out[t0 : t0 + qlen] - ref)) < 1e-12
+
+
+# ---- per-tensor quantisation of Q (Section 3.8: Q, K and V each share one scalar scale) ----
+
+def _q_image_bits(q_bits, q_scale):
+    """bf16 bit patterns of e4m3(float32(q) * float32(1/q_scale)), the E4M3 image of Q WITHOUT its
+    scale, computed with torch's own float8 conversion (every E4M3 value is exact in bf16)."""
+    qf = _f64(q_bits).float()
+    inv = float(np.float32(1.0) / np.float32(q_scale))
+    img = (qf * inv).clamp(-448, 448).to(torch.float8_e4m3fn).float()
+    return img.to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+
+
+@pytest.mark.parametrize("case", CASES)
+@pytest.mark.parametrize("q_scale", [0.0625, 0.03, 0.011])
+def test_quantised_q_equals_the_unquantised_oracle_on_the_e4m3_image_of_q(case, q_scale):
+    """With q_scale set the oracle must give what it gives without it on Q replaced by its E4M3 image
+    (made by torch, not by the oracle) with the scale of Q folded into the softmax scale.  Pins the
+    conversion, the place where the scale enters and that nothing but the scores sees it."""
+    ql, kl, hq, hkv, d, ps = case
+    meta = wl.build_meta("fp8q", ql, kl, num_q_heads=hq, num_kv_heads=hkv, head_dim=d, page_size=ps, seed=19,
+                         kv_fp8=True, k_scale=0.023, v_scale=0.031)
+    batch = wl.materialize(meta)
+    args = (wl.bf16_bits(batch.new_k), wl.bf16_bits(batch.new_v))
+    base = dict(num_q_heads=hq, num_kv_heads=hkv, head_dim=d, page_size=ps, num_pages=meta.num_pages,
+                max_pages_per_seq=meta.max_pages_per_seq, causal=True, kv_fp8=True, k_scale=meta.k_scale, v_scale=meta.v_scale)
+    q_bits = wl.bf16_bits(batch.q)
+    cache_a, cache_b = wl.bf16_bits(batch.kv_cache).copy(), wl.bf16_bits(batch.kv_cache).copy()
+    got = orc.forward(orc.OracleShape(scale=meta.sm_scale, q_scale=q_scale, **base), q_bits, *args, cache_a,
+                      meta.page_table, meta.cu_q_lens, meta.kv_lens)
+    folded = meta.sm_scale * float(np.float32(q_scale))
+    want = orc.forward(orc.OracleShape(scale=folded, q_scale=0.0, **base), _q_image_bits(q_bits, q_scale), *args, cache_b,
+                       meta.page_table, meta.cu_q_lens, meta.kv_lens)
+    assert np.array_equal(cache_a, cache_b)  # the cache update does not depend on the scale of Q
+    assert np.max(np.abs(got - want)) < 1e-12
+    # and it differs from the bf16-Q result by what E4M3's 3 mantissa bits allow, no more: a dropped
+    # quantisation (or a scale applied twice) fails one of the two bounds
+    cache_c = wl.bf16_bits(batch.kv_cache).copy()
+    plain = orc.forward(orc.OracleShape(scale=meta.sm_scale, q_scale=0.0, **base), q_bits, *args, cache_c,
+                        meta.page_table, meta.cu_q_lens, meta.kv_lens)
+    diff = np.abs(got - plain)
+    assert 1e-6 < diff.max() < 0.5
+
+
+def test_q_scale_is_rejected_without_an_fp8_cache_and_when_negative():
+    meta = wl.build_meta("fp8q-bad", [2], [9], num_q_heads=4, num_kv_heads=2, head_dim=32, page_size=8, seed=20)
+    batch = wl.materialize(meta)
+    base = dict(num_q_heads=4, num_kv_heads=2, head_dim=32, page_size=8, num_pages=meta.num_pages,
+                max_pages_per_seq=meta.max_pages_per_seq, scale=meta.sm_scale)
+    with pytest.raises(ValueError):
+        orc.forward(orc.OracleShape(q_scale=0.05, **base), wl.bf16_bits(batch.q), wl.bf16_bits(batch.new_k),
+                    wl.bf16_bits(batch.new_v), wl.bf16_bits(batch.kv_cache).copy(), meta.page_table, meta.cu_q_lens,
+                    meta.kv_lens)
+
+
+def test_q_saturates_at_the_largest_e4m3_value():
+    """A query element beyond 448 * q_scale is clamped, as K and V are: with a single key the output
+    is that key's value whatever Q is, so use two keys whose scores differ only through the clamp."""
+    hq = hkv = 1
+    d, ps = 16, 8
+    meta = wl.build_meta("fp8q-sat", [1], [2], num_q_heads=hq, num_kv_heads=hkv, head_dim=d, page_size=ps, seed=21,
+                         kv_fp8=True, k_scale=1.0, v_scale=1.0)
+    q = torch.zeros(1, 1, d)
+    q[0, 0, 0] = 1000.0  # far beyond 448 * q_scale
+    to_bits = lambda t: t.to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    k_new = torch.zeros(1, 1, d); k_new[0, 0, 0] = 1.0
+    v_new = torch.ones(1, 1, d)
+    cache = np.zeros((meta.num_pages, ps, 2, d), np.uint8)  # cached key 0 = 0 -> score 0; value 0
+    shape = orc.OracleShape(hq, hkv, d, ps, meta.num_pages, meta.max_pages_per_seq, 0.01, True, True, 1.0, 1.0, 1.0)
+    out = orc.forward(shape, to_bits(q), to_bits(k_new), to_bits(v_new), cache, meta.page_table, meta.cu_q_lens, meta.kv_lens)
+    # scores: key 0 -> 0, key 1 -> 0.01 * 448 * 1 (clamped), not 0.01 * 1000; value 1 for key 1, 0 for key 0
+    w = np.exp(0.01 * 448.0)
+    assert abs(out[0, 0, 0] - w / (1.0 + w)) < 1e-12
