@@ -207,7 +207,7 @@ def oracle_sample(meta, batch, budget_s: float = 15.0, rate: float | None = None
     pick.sort()
     host, n_pages, _, _ = wl.host_subset(batch, pick)
     shape = orc.OracleShape(meta.num_q_heads, meta.num_kv_heads, meta.head_dim, meta.page_size, n_pages,
-                            meta.max_pages_per_seq, meta.sm_scale, meta.causal, meta.kv_fp8, meta.k_scale, meta.v_scale)
+                            meta.max_pages_per_seq, meta.sm_scale, meta.causal, meta.kv_fp8, meta.k_scale, meta.v_scale, meta.q_scale)
     triples = [(k, i, a) for k, r in enumerate(pick) for i in range(int(meta.q_lens[r])) for a in range(meta.num_q_heads)]
     frac = 1.0
     if acc > 1.5 * budget_s * rate:  # a single request may still be too long (full prefill): sample its rows
@@ -336,6 +336,9 @@ def run_leg(workload, args, rank, world, local, dist, peaks):
     if args.kv_fp8:
         meta.kv_fp8, meta.k_scale, meta.v_scale = True, 0.02, 0.02
         meta.name += "_fp8kv"
+        if args.q_fp8:
+            meta.q_scale = 0.02
+            meta.name += "q"
     batch = wl.materialize(meta, device)
     rapi = binding.Rpa.for_meta(meta, device=local)
     if args.kv_chunk:
@@ -566,6 +569,7 @@ def main():
     ap.add_argument("--noncausal", action="store_true", help="paper_* workloads without the causal mask")
     ap.add_argument("--head-dim", type=int, default=128, help="head dimension of the paper_* workloads (128 or 256)")
     ap.add_argument("--kv-fp8", action="store_true", help="FP8 E4M3 cache with per-tensor scales (decode workloads)")
+    ap.add_argument("--q-fp8", action="store_true", help="with --kv-fp8: Q is quantised to E4M3 with a per-tensor scale as well")
     ap.add_argument("--plan", default="host", choices=["host", "device"],
                     help="who builds the work lists each step: rpa_plan on the host, or rpa_plan_device on the GPU")
     ap.add_argument("--shard", default="requests", choices=["requests", "heads"],

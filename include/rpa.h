@@ -34,7 +34,9 @@
  * Quantised cache (the paper's per-tensor quantisation, Section 3.8).  With kv_dtype =
  * RPA_KV_FP8_E4M3 a cache element is one FP8 E4M3 byte that stands for byte_value * k_scale (K) or
  * byte_value * v_scale (V); kv_cache is then [num_pages, page_size, 2*h_kv, d_k] bytes.  q, new_k,
- * new_v and out stay bf16.  The update stores e4m3(float(x) * (1/scale)) (fp32 multiply by the fp32
+ * new_v and out stay bf16 at the boundary.  With q_scale > 0 the queries are taken in E4M3 precision
+ * as well, each element as e4m3(float(q) * (1/q_scale)) * q_scale (the conversion K uses; a pass over
+ * the call's T query rows that precedes the attention kernels).  The update stores e4m3(float(x) * (1/scale)) (fp32 multiply by the fp32
  * reciprocal, round to nearest even, saturating at +-448), and attention sees every key and value,
  * the batch's own new tokens included, in that quantised precision.  With head_dim 128 or 256
  * long queries run on the tensor-core tile kernels as with a bf16 cache (their new tokens are
@@ -98,6 +100,8 @@ typedef struct {
     int32_t kv_dtype;          /* RPA_KV_BF16 (0) or RPA_KV_FP8_E4M3 (1)                            */
     float k_scale;             /* FP8 cache: per-tensor scales (Section 3.8); ignored for bf16      */
     float v_scale;
+    float q_scale;             /* FP8 cache only: > 0 quantises Q to E4M3 with this per-tensor scale
+                                  too (Section 3.8); 0 leaves Q in bf16                              */
 } rpa_config_t;
 
 typedef struct {

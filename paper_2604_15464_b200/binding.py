@@ -41,7 +41,7 @@ class rpa_config_t(ctypes.Structure):
                 ("page_size", ctypes.c_int32), ("num_pages", ctypes.c_int32), ("max_pages_per_seq", ctypes.c_int32),
                 ("max_num_seqs", ctypes.c_int32), ("max_num_tokens", ctypes.c_int32), ("sm_scale", ctypes.c_float),
                 ("causal", ctypes.c_int32), ("kv_dtype", ctypes.c_int32), ("k_scale", ctypes.c_float),
-                ("v_scale", ctypes.c_float)]
+                ("v_scale", ctypes.c_float), ("q_scale", ctypes.c_float)]
 
 
 class rpa_plan_info_t(ctypes.Structure):
@@ -115,11 +115,12 @@ class RpaConfig:
     kv_fp8: bool = False  # FP8 E4M3 cache with per-tensor scales
     k_scale: float = 1.0
     v_scale: float = 1.0
+    q_scale: float = 0.0  # > 0: Q is quantised to E4M3 with this per-tensor scale as well (FP8 cache only)
 
     def _c(self) -> rpa_config_t:
         return rpa_config_t(self.num_q_heads, self.num_kv_heads, self.head_dim, self.page_size, self.num_pages,
                             self.max_pages_per_seq, self.max_num_seqs, self.max_num_tokens, self.sm_scale,
-                            1 if self.causal else 0, 1 if self.kv_fp8 else 0, self.k_scale, self.v_scale)
+                            1 if self.causal else 0, 1 if self.kv_fp8 else 0, self.k_scale, self.v_scale, self.q_scale)
 
 
 def _dev_ptr(t) -> int:
@@ -167,7 +168,7 @@ class Rpa:
         """Handle sized for a ``workloads.BatchMeta``."""
         cfg = RpaConfig(meta.num_q_heads, meta.num_kv_heads, meta.head_dim, meta.page_size, meta.num_pages,
                         meta.max_pages_per_seq, max(meta.num_seqs, 1), max(meta.token_capacity, 1), meta.scale,
-                        meta.causal, meta.kv_fp8, meta.k_scale, meta.v_scale)
+                        meta.causal, meta.kv_fp8, meta.k_scale, meta.v_scale, getattr(meta, "q_scale", 0.0))
         library_path = over.pop("library_path", None)
         for k, v in over.items():
             setattr(cfg, k, v)

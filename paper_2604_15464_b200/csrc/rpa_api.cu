@@ -69,6 +69,8 @@ struct rpa_handle {
     int32_t* d_dev_scratch = nullptr;
     int32_t dev_hist_len = 0;
     uint16_t* d_new_codes = nullptr;  // FP8 cache with a tile path: bf16 copies of new_k | new_v after quantisation
+    uint16_t* d_q_img = nullptr;      // quantised Q (q_scale > 0): the E4M3 values of the call's query rows as bf16 ...
+    uint8_t* d_q_codes = nullptr;     // ... and their codes
     float* d_partial_o = nullptr;
     float* d_partial_ml = nullptr;
     uint32_t* d_status = nullptr;
@@ -109,6 +111,7 @@ bool valid_config(const rpa_config_t& c, rpa_status_t* why) {
     if (c.max_num_seqs <= 0 || c.max_num_tokens <= 0 || !(c.sm_scale >= 0.f)) return false;
     if (c.kv_dtype != RPA_KV_BF16 && c.kv_dtype != RPA_KV_FP8_E4M3) return false;
     if (c.kv_dtype == RPA_KV_FP8_E4M3 && !(c.k_scale > 0.f && c.v_scale > 0.f)) return false;
+    if (!(c.q_scale >= 0.f) || (c.q_scale > 0.f && c.kv_dtype != RPA_KV_FP8_E4M3)) return false;  // a scale for Q goes with an FP8 cache
     *why = RPA_ERR_UNSUPPORTED;
     if (!row_kernel_supported(c.head_dim, c.num_q_heads / c.num_kv_heads)) return false;
     if (c.page_size % kKvTile) return false;
@@ -133,6 +136,8 @@ void free_all(rpa_handle* h) {
         cudaFree(h->d_group_counters);
         cudaFree(h->d_partial_o);
         cudaFree(h->d_new_codes);
+        cudaFree(h->d_q_img);
+        cudaFree(h->d_q_codes);
         for (int b = 0; b < 2; ++b) {
             cudaFree(h->d_dev_lists_buf[b]);
             cudaFree(h->d_dev_counts_buf[b]);
@@ -304,6 +309,11 @@ rpa_status_t rpa_create(const rpa_config_t* cfg, int device, rpa_handle_t** out)
         }
         if (e == cudaSuccess && cfg->kv_dtype == RPA_KV_FP8_E4M3 && p.tile_min_q > 0)
             e = cudaMalloc(&h->d_new_codes, (size_t)2 * cfg->max_num_tokens * cfg->num_kv_heads * cfg->head_dim * sizeof(uint16_t));
+        if (e == cudaSuccess && cfg->q_scale > 0.f) {
+            const size_t q_elems = (size_t)cfg->max_num_tokens * cfg->num_q_heads * cfg->head_dim;
+            e = cudaMalloc(&h->d_q_img, q_elems * sizeof(uint16_t));
+            if (e == cudaSuccess) e = cudaMalloc(&h->d_q_codes, q_elems);
+        }
         if (e == cudaSuccess) e = cudaMalloc(&h->d_group_counters, (size_t)p.max_groups * sizeof(int32_t));
         if (e == cudaSuccess) e = cudaMemset(h->d_group_counters, 0, (size_t)p.max_groups * sizeof(int32_t));
         if (e == cudaSuccess)
@@ -383,7 +393,8 @@ static KernelArgs common_kernel_args(const rpa_handle* h, uint8_t* lists, size_t
                                      const int32_t* kv_lens, void* out) {
     const rpa_config_t& c = h->cfg;
     KernelArgs a{};
-    a.q = static_cast<const uint16_t*>(q);
+    // with a scale for Q the kernels read the quantised image the pass before them has made
+    a.q = c.q_scale > 0.f ? h->d_q_img : static_cast<const uint16_t*>(q);
     a.new_k = static_cast<const uint16_t*>(new_k);
     a.new_v = static_cast<const uint16_t*>(new_v);
     a.kv_cache = static_cast<uint16_t*>(kv_cache);
@@ -409,7 +420,7 @@ static KernelArgs common_kernel_args(const rpa_handle* h, uint8_t* lists, size_t
     a.causal = c.causal ? 1 : 0;
     const bool fp8 = c.kv_dtype == RPA_KV_FP8_E4M3;
     a.kv_fp8 = fp8 ? 1 : 0;
-    a.scale_log2 = c.sm_scale * 1.4426950408889634f * (fp8 ? c.k_scale : 1.f);
+    a.scale_log2 = c.sm_scale * 1.4426950408889634f * (fp8 ? c.k_scale : 1.f) * (c.q_scale > 0.f ? c.q_scale : 1.f);
     a.out_scale = fp8 ? c.v_scale : 1.f;
     a.inv_k_scale = fp8 ? 1.0f / c.k_scale : 1.f;
     a.inv_v_scale = fp8 ? 1.0f / c.v_scale : 1.f;
@@ -440,6 +451,9 @@ static rpa_status_t forward_device_planned(rpa_handle* h, const void* q, const v
     const int b = h->dev_cur;
     const bool capturing = stream_is_capturing(s);
     if (!capturing && h->dev_planned_pending[b]) RPA_CUDA(h, cudaStreamWaitEvent(s, h->ev_dev_planned[b], 0));  // the plan may come from another stream
+    if (c.q_scale > 0.f)  // (T is known on the device only: the pass bounds its rows by cu_q_lens[num_seqs])
+        RPA_CUDA(h, launch_quantise_q(static_cast<const uint16_t*>(q), h->d_q_img, h->d_q_codes, 0, cu_q_lens, h->planned_num_seqs,
+                                      c.max_num_tokens, c.num_q_heads * c.head_dim, 1.0f / c.q_scale, h->d_status, true, s));
     const bool tiles = h->policy.tile_min_q > 0;
     const bool single_tile = tile1_kernel_supported(c.head_dim, c.num_q_heads / c.num_kv_heads);
     // eight waves of resident CTAs: short lists get one item per CTA (placed dynamically by the
@@ -645,6 +659,10 @@ rpa_status_t rpa_forward(rpa_handle_t* h, const void* q, const void* new_k, cons
         a.validated = 1;
         RPA_CUDA(h, launch_validate_kernel(a, num_seqs, reinterpret_cast<const int32_t*>(lists + h->buf_off_kvlens[h->cur]), s));
     }
+    if (h->cfg.q_scale > 0.f)
+        RPA_CUDA(h, launch_quantise_q(static_cast<const uint16_t*>(q), h->d_q_img, h->d_q_codes, h->plan.info.num_tokens, nullptr, 0,
+                                      h->cfg.max_num_tokens, h->cfg.num_q_heads * h->cfg.head_dim, 1.0f / h->cfg.q_scale, h->d_status,
+                                      h->validate, s));
     const bool single_tile = tile1_kernel_supported(h->cfg.head_dim, h->cfg.num_q_heads / h->cfg.num_kv_heads);
     const bool side_by_side = a.num_row_items > 0 && a.num_tile_items > 0 && !(h->ablation & kAblateOverlap);
     if (side_by_side) {

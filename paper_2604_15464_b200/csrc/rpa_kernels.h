@@ -106,6 +106,11 @@ int row_kernel_fp8_ctas_per_sm(int head_dim);
 int row_kernel_fp8_narrow_ctas_per_sm(int head_dim);  // the 8-row instantiation, chosen when no row item has more rows
 cudaError_t row_kernel_fp8_prepare(int head_dim, int group);
 cudaError_t launch_row_kernel_fp8(const KernelArgs& a, cudaStream_t stream);
+// per-tensor quantisation of Q (Section 3.8): q -> bf16 images of its E4M3 values and the raw codes; the rows are
+// bounded by total_rows, or, when cu_q_lens (device) is given, by cu_q_lens[num_seqs] (at most max_rows)
+cudaError_t launch_quantise_q(const uint16_t* q, uint16_t* q_img, uint8_t* q_codes, int64_t total_rows, const int32_t* cu_q_lens,
+                              int32_t num_seqs, int64_t max_rows, int32_t row_elems, float inv_q_scale, const uint32_t* status,
+                              bool check_status, cudaStream_t stream);
 
 // The tensor maps of a tile-kernel launch, kept from launch to launch: encoding the five maps costs
 // several microseconds of host time, and a serving loop passes the same tensors step after step.  An

@@ -298,7 +298,8 @@ rpa_status_t build_plan(const rpa_config_t& cfg, const PlanPolicy& policy, const
     info.kv_chunk_tokens = (int32_t)std::min<int64_t>(chunk, INT_MAX);
     // (an FP8 cache adds the quantising pass that runs before the tile kernel)
     info.gpu_launches = (plan.rows.empty() ? 0 : 1) + (plan.tiles.empty() ? 0 : cfg.kv_dtype == RPA_KV_FP8_E4M3 ? 2 : 1) +
-                        ((plan.groups.empty() || policy.fused_combine) ? 0 : 1);
+                        ((plan.groups.empty() || policy.fused_combine) ? 0 : 1) +
+                        ((cfg.q_scale > 0.f && T > 0) ? 1 : 0);  // the pass that quantises Q
     info.algorithmic_bytes = bytes;
     info.algorithmic_flops = 4 * (int64_t)cfg.num_q_heads * cfg.head_dim * pairs;
     // SM split for mixed batches: the tile kernel is persistent on tile_ctas SMs while row items

@@ -1,3 +1,4 @@
+#include <algorithm>
 // Split-KV row kernel on an FP8 (E4M3) cache with per-tensor scales (the paper's Section 3.8).
 //
 // Same work items, ring structure, softmax and merge as rpa_row_kernel.cu; what changes is the data
@@ -585,6 +586,45 @@ cudaError_t launch_row_kernel_fp8_strided(const KernelArgs& a, int grid, bool na
     if (grid <= 0 || !a.dev_counts) return cudaErrorInvalidValue;
     RPA_DISPATCH_DG8(a.head_dim, a.h_q / a.h_kv, launch_row8_strided, a, grid, narrow, stream);
     return cudaErrorInvalidValue;
+}
+
+// Per-tensor quantisation of Q (Section 3.8): every element of the call's query rows becomes
+// e4m3(float(q) * (1/q_scale)), the conversion K uses.  The pass writes the E4M3 VALUES as bf16 (each
+// is exact in bf16) into a scratch tensor the attention kernels then read in place of q, with q_scale
+// folded into the softmax scale, and the raw codes beside them.  `total_rows` bounds the rows when
+// the host knows T; with a device-made plan the bound is cu_q_lens[num_seqs], read on the device.
+__global__ void __launch_bounds__(256) rpa_quantise_q_kernel(const uint16_t* q, uint16_t* q_img, uint8_t* q_codes, int64_t total_rows,
+                                                             const int32_t* cu_q_lens, int32_t num_seqs, int32_t row_elems,
+                                                             float inv_q_scale, const uint32_t* status, int32_t check_status) {
+    if (check_status && (*reinterpret_cast<const volatile uint32_t*>(status) & kStatusBadInput)) return;
+    const int64_t rows = cu_q_lens ? (int64_t)cu_q_lens[num_seqs] : total_rows;
+    const int64_t n16 = rows * row_elems / 16;  // (row_elems is a multiple of 64)
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n16; i += (int64_t)gridDim.x * blockDim.x) {
+        const uint4 codes = quantise16(q + i * 16, inv_q_scale);
+        *reinterpret_cast<uint4*>(q_codes + i * 16) = codes;
+        uint4 lo, hi;
+        lo.x = e4m3x2_to_bf16x2(codes.x & 0xffffu);
+        lo.y = e4m3x2_to_bf16x2(codes.x >> 16);
+        lo.z = e4m3x2_to_bf16x2(codes.y & 0xffffu);
+        lo.w = e4m3x2_to_bf16x2(codes.y >> 16);
+        hi.x = e4m3x2_to_bf16x2(codes.z & 0xffffu);
+        hi.y = e4m3x2_to_bf16x2(codes.z >> 16);
+        hi.z = e4m3x2_to_bf16x2(codes.w & 0xffffu);
+        hi.w = e4m3x2_to_bf16x2(codes.w >> 16);
+        *reinterpret_cast<uint4*>(q_img + i * 16) = lo;
+        *reinterpret_cast<uint4*>(q_img + i * 16 + 8) = hi;
+    }
+}
+
+cudaError_t launch_quantise_q(const uint16_t* q, uint16_t* q_img, uint8_t* q_codes, int64_t total_rows, const int32_t* cu_q_lens,
+                              int32_t num_seqs, int64_t max_rows, int32_t row_elems, float inv_q_scale, const uint32_t* status,
+                              bool check_status, cudaStream_t stream) {
+    const int64_t n16 = (cu_q_lens ? max_rows : total_rows) * row_elems / 16;
+    if (n16 <= 0) return cudaSuccess;
+    const int grid = (int)std::min<int64_t>((n16 + 255) / 256, 148 * 16);
+    rpa_quantise_q_kernel<<<grid, 256, 0, stream>>>(q, q_img, q_codes, total_rows, cu_q_lens, num_seqs, row_elems, inv_q_scale, status,
+                                                    check_status ? 1 : 0);
+    return cudaGetLastError();
 }
 
 cudaError_t launch_row_kernel_fp8(const KernelArgs& a, cudaStream_t stream) {

@@ -48,6 +48,7 @@ class BatchMeta:
     kv_fp8: bool = False  # FP8 E4M3 cache with per-tensor scales (the paper's Section 3.8)
     k_scale: float = 1.0
     v_scale: float = 1.0
+    q_scale: float = 0.0  # > 0: Q is quantised to E4M3 with this per-tensor scale as well (FP8 cache only)
 
     @property
     def num_seqs(self) -> int:
@@ -95,7 +96,7 @@ def build_meta(name: str, q_lens: Sequence[int], kv_lens: Sequence[int], *, num_
                head_dim: int, page_size: int, num_pages: Optional[int] = None, pool_slack: float = 1.25,
                token_capacity: Optional[int] = None, causal: bool = True, scale: float = 0.0, seed: int = 0,
                max_pages_per_seq: Optional[int] = None, kv_fp8: bool = False, k_scale: float = 1.0,
-               v_scale: float = 1.0) -> BatchMeta:
+               v_scale: float = 1.0, q_scale: float = 0.0) -> BatchMeta:
     """Lay the requests out on randomly permuted physical pages of a pool of ``num_pages`` pages."""
     q_lens = np.asarray(q_lens, dtype=np.int32)
     kv_lens = np.asarray(kv_lens, dtype=np.int32)
@@ -121,7 +122,7 @@ def build_meta(name: str, q_lens: Sequence[int], kv_lens: Sequence[int], *, num_
     cap = int(q_lens.sum()) if token_capacity is None else int(token_capacity)
     assert cap >= int(q_lens.sum())
     return BatchMeta(name, num_q_heads, num_kv_heads, head_dim, page_size, int(num_pages), int(max_pages_per_seq),
-                     q_lens, kv_lens, table, max(cap, 1), causal, scale, seed, kv_fp8, k_scale, v_scale)
+                     q_lens, kv_lens, table, max(cap, 1), causal, scale, seed, kv_fp8, k_scale, v_scale, q_scale)
 
 
 LLAMA3_8B = dict(num_q_heads=32, num_kv_heads=8, head_dim=128)

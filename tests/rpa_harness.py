@@ -18,7 +18,7 @@ SENTINEL = 0x7FC1  # a NaN pattern no computation produces; marks rows the call 
 def oracle_shape(meta, num_pages=None):
     return orc.OracleShape(meta.num_q_heads, meta.num_kv_heads, meta.head_dim, meta.page_size,
                            meta.num_pages if num_pages is None else num_pages, meta.max_pages_per_seq, meta.sm_scale,
-                           meta.causal, meta.kv_fp8, meta.k_scale, meta.v_scale)
+                           meta.causal, meta.kv_fp8, meta.k_scale, meta.v_scale, meta.q_scale)
 
 
 def bf16_to_f64(bits: np.ndarray) -> np.ndarray:

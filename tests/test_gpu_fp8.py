@@ -178,3 +178,50 @@ def test_fp8_narrow_noncausal_and_wide_beside_it():
         meta = wl.build_meta("fp8nw", [1, 3, 1], [500, 90, 33], num_q_heads=32, num_kv_heads=8, head_dim=128,
                              page_size=16, seed=43, kv_fp8=True, k_scale=0.03, v_scale=0.03)
         hz.full_parity(wl.materialize(meta, _dev(), canaries=True), tile_min_q=10**6, device_plan=device_plan)
+
+
+# ---- per-tensor quantisation of Q as well (Section 3.8): the oracle takes Q in E4M3 precision ----
+
+QFP8_CASES = [
+    # q_lens, kv_lens, h_q, h_kv, d, page_size, tile_min_q
+    ([1, 1, 12, 5], [33, 7, 12, 29], 4, 2, 64, 16, None),           # row kernel, d = 64
+    ([1] * 9, [5, 31, 32, 33, 47, 48, 49, 255, 257], 32, 8, 128, 128, None),  # decode rows (8-row instantiation)
+    ([3, 0, 1, 40, 17], [3, 0, 130, 40, 100], 32, 8, 128, 16, None),          # default routing: rows and tiles
+    ([200, 1, 70], [200, 500, 1000], 32, 8, 128, 16, 1),             # everything on the tile kernel
+    ([16, 32, 5], [1016, 2080, 133], 32, 8, 128, 16, 1),             # short items split over both accumulators
+    ([1, 4, 40], [700, 64, 300], 32, 8, 256, 16, 1),                 # d = 256: the single-tile kernel
+    ([5, 9, 1], [21, 9, 300], 8, 1, 128, 16, 10 ** 6),               # MQA on the 16-row instantiation
+]
+
+
+@pytest.mark.parametrize("case", QFP8_CASES)
+@pytest.mark.parametrize("device_plan", [False, True])
+def test_fp8_cache_with_quantised_q(case, device_plan):
+    ql, kl, hq, hkv, d, ps, tile_min_q = case
+    meta = wl.build_meta("fp8q", ql, kl, num_q_heads=hq, num_kv_heads=hkv, head_dim=d, page_size=ps, seed=29,
+                         token_capacity=sum(ql) + 3, kv_fp8=True, k_scale=0.023, v_scale=0.031, q_scale=0.027)
+    if device_plan and tile_min_q is not None:
+        pytest.skip("the routing threshold is a host-planner knob in this test")
+    hz.full_parity(wl.materialize(meta, _dev(), canaries=True), tile_min_q=tile_min_q, device_plan=device_plan)
+
+
+def test_quantised_q_really_is_quantised():
+    """The same batch with and without a scale for Q must differ (by what three mantissa bits allow):
+    a pass that were skipped, or a scale that were not folded, would show here or in the parity above."""
+    shape = dict(num_q_heads=32, num_kv_heads=8, head_dim=128, page_size=16, seed=30, kv_fp8=True, k_scale=0.023, v_scale=0.031)
+    a = wl.build_meta("fp8q-a", [1, 40], [300, 200], **shape)
+    b = wl.build_meta("fp8q-b", [1, 40], [300, 200], q_scale=0.027, **shape)
+    out_a, _ = hz.run_gpu(wl.materialize(a, _dev()))
+    out_b, _ = hz.run_gpu(wl.materialize(b, _dev()))
+    diff = np.abs(hz.bf16_to_f64(out_a[: a.num_tokens]) - hz.bf16_to_f64(out_b[: b.num_tokens]))
+    assert 1e-4 < diff.max() < 0.5
+
+
+def test_q_scale_needs_an_fp8_cache():
+    from paper_2604_15464_b200 import binding
+
+    meta = wl.build_meta("q-bf16", [1], [40], num_q_heads=32, num_kv_heads=8, head_dim=128, page_size=16, seed=31)
+    meta.q_scale = 0.05
+    with pytest.raises(binding.RpaError) as err:
+        binding.Rpa.for_meta(meta)
+    assert err.value.status == 1  # RPA_ERR_INVALID_ARG

@@ -23,7 +23,7 @@ pytestmark = pytest.mark.gpu
 def _config(meta):
     return binding.RpaConfig(meta.num_q_heads, meta.num_kv_heads, meta.head_dim, meta.page_size, meta.num_pages,
                              meta.max_pages_per_seq, max(meta.num_seqs, 1), max(meta.token_capacity, 1), meta.scale,
-                             meta.causal, meta.kv_fp8, meta.k_scale, meta.v_scale)
+                             meta.causal, meta.kv_fp8, meta.k_scale, meta.v_scale, meta.q_scale)
 
 
 def _run_static(meta, stream=None):
