@@ -71,6 +71,7 @@ struct rpa_handle {
     uint16_t* d_new_codes = nullptr;  // FP8 cache with a tile path: bf16 copies of new_k | new_v after quantisation
     uint16_t* d_q_img = nullptr;      // quantised Q (q_scale > 0): the E4M3 values of the call's query rows as bf16 ...
     uint8_t* d_q_codes = nullptr;     // ... and their codes
+    uint8_t* d_new_k_codes8 = nullptr;  // ... and, for the FP8 score product of the tile kernel, the K codes of the call's own tokens
     float* d_partial_o = nullptr;
     float* d_partial_ml = nullptr;
     uint32_t* d_status = nullptr;
@@ -138,6 +139,7 @@ void free_all(rpa_handle* h) {
         cudaFree(h->d_new_codes);
         cudaFree(h->d_q_img);
         cudaFree(h->d_q_codes);
+        cudaFree(h->d_new_k_codes8);
         for (int b = 0; b < 2; ++b) {
             cudaFree(h->d_dev_lists_buf[b]);
             cudaFree(h->d_dev_counts_buf[b]);
@@ -313,6 +315,8 @@ rpa_status_t rpa_create(const rpa_config_t* cfg, int device, rpa_handle_t** out)
             const size_t q_elems = (size_t)cfg->max_num_tokens * cfg->num_q_heads * cfg->head_dim;
             e = cudaMalloc(&h->d_q_img, q_elems * sizeof(uint16_t));
             if (e == cudaSuccess) e = cudaMalloc(&h->d_q_codes, q_elems);
+            if (e == cudaSuccess && cfg->head_dim == 128 && p.tile_min_q > 0)
+                e = cudaMalloc(&h->d_new_k_codes8, (size_t)cfg->max_num_tokens * cfg->num_kv_heads * cfg->head_dim);
         }
         if (e == cudaSuccess) e = cudaMalloc(&h->d_group_counters, (size_t)p.max_groups * sizeof(int32_t));
         if (e == cudaSuccess) e = cudaMemset(h->d_group_counters, 0, (size_t)p.max_groups * sizeof(int32_t));
@@ -398,6 +402,9 @@ static KernelArgs common_kernel_args(const rpa_handle* h, uint8_t* lists, size_t
     a.new_k = static_cast<const uint16_t*>(new_k);
     a.new_v = static_cast<const uint16_t*>(new_v);
     a.kv_cache = static_cast<uint16_t*>(kv_cache);
+    a.q_codes = h->d_q_codes;
+    a.new_k_codes8 = h->d_new_k_codes8;
+    a.q_fp8 = h->d_new_k_codes8 != nullptr && !(h->ablation & 16u) ? 1 : 0;  // (ablation bit 4: bf16 score products on the images instead)
     a.new_k_codes = h->d_new_codes;
     a.new_v_codes = h->d_new_codes ? h->d_new_codes + (size_t)c.max_num_tokens * c.num_kv_heads * c.head_dim : nullptr;
     a.page_table = page_table;

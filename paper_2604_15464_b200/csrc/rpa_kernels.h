@@ -19,6 +19,12 @@ struct KernelArgs {
     uint16_t* kv_cache;
     uint16_t* new_k_codes;  // FP8 cache, tile path: scratch copies of new_k / new_v holding the values of
     uint16_t* new_v_codes;  // the quantised codes as bf16 (written by the pass before the tile kernel)
+    // Quantised Q (a per-tensor scale for Q as well) on the d_k = 128 tile path: the score product runs
+    // on the FP8 tensor-core format straight on code bytes - the E4M3 codes of the call's query rows and,
+    // for the batch's own tokens, a scratch copy of their K codes (context keys are the cache's bytes).
+    const uint8_t* q_codes;  // [T, h_q, d]
+    uint8_t* new_k_codes8;   // [T, h_kv, d]
+    int32_t q_fp8;           // 1: the tile kernel takes Q and K as E4M3 codes
     const int32_t* page_table;
     const int32_t* cu_q_lens;
     const int32_t* kv_lens;
@@ -122,7 +128,7 @@ struct TileMapCache {
         bool valid = false;
         const void *q = nullptr, *out = nullptr, *new_k = nullptr, *new_v = nullptr, *kv_cache = nullptr;
         int64_t token_rows = 0;
-        int32_t h_q = 0, h_kv = 0, head_dim = 0, page_size = 0, num_pages = 0, kv_fp8 = 0, block_n = 0, q_tile_tokens = 0;
+        int32_t h_q = 0, h_kv = 0, head_dim = 0, page_size = 0, num_pages = 0, kv_fp8 = 0, q_fp8 = 0, block_n = 0, q_tile_tokens = 0;
         alignas(64) unsigned char maps[5 * 128];  // five CUtensorMap objects (128 bytes each)
     } entries[kEntries];
     int next = 0;

@@ -204,6 +204,7 @@ __global__ void __launch_bounds__(128) rpa_quantise_new_kernel(const KernelArgs 
         }
         const int64_t src = (((int64_t)cu + tok) * a.h_kv + it.kv_head) * D + piece * 16;
         const uint4 codes = quantise16((kv ? a.new_v : a.new_k) + src, kv ? a.inv_v_scale : a.inv_k_scale);
+        if (!kv && a.new_k_codes8) *reinterpret_cast<uint4*>(a.new_k_codes8 + src) = codes;  // for the FP8 score product
         if (!(a.ablation & kAblateUpdate)) {
             const int page = pt[pos / a.page_size];
             if (debug_write_page_ok(a, page))
@@ -276,7 +277,13 @@ inline bool build_tile_maps(const KernelArgs& a, int64_t token_rows, int D, int 
         const uint64_t dims[3] = {d, (uint64_t)a.h_q, (uint64_t)token_rows};
         const uint64_t str[2] = {d * 2, d * 2 * a.h_q};
         const uint32_t box[3] = {64, (uint32_t)G, (uint32_t)q_tile_tokens};
-        if (!make_map(&maps->q, a.q, 3, dims, str, box)) return false;
+        if (a.q_fp8) {  // code bytes: a row of 128 codes is one 128-byte swizzle span
+            const uint64_t str8[2] = {d, d * a.h_q};
+            const uint32_t box8[3] = {128, (uint32_t)G, (uint32_t)q_tile_tokens};
+            if (D != 128 || !make_map(&maps->q, a.q_codes, 3, dims, str8, box8, CU_TENSOR_MAP_DATA_TYPE_UINT8)) return false;
+        } else if (!make_map(&maps->q, a.q, 3, dims, str, box)) {
+            return false;
+        }
         if (!make_map(&maps->out, a.out, 3, dims, str, box)) return false;
     }
     {
@@ -284,7 +291,13 @@ inline bool build_tile_maps(const KernelArgs& a, int64_t token_rows, int D, int 
         const uint64_t str[2] = {d * 2, d * 2 * a.h_kv};
         const uint32_t box[3] = {64, 1, (uint32_t)block_n};
         // FP8 cache: the new-token key blocks come from the scratch copies that hold the quantised values
-        if (!make_map(&maps->new_k, a.kv_fp8 ? a.new_k_codes : a.new_k, 3, dims, str, box)) return false;
+        if (a.q_fp8) {
+            const uint64_t str8[2] = {d, d * a.h_kv};
+            const uint32_t box8[3] = {128, 1, (uint32_t)block_n};
+            if (!make_map(&maps->new_k, a.new_k_codes8, 3, dims, str8, box8, CU_TENSOR_MAP_DATA_TYPE_UINT8)) return false;
+        } else if (!make_map(&maps->new_k, a.kv_fp8 ? a.new_k_codes : a.new_k, 3, dims, str, box)) {
+            return false;
+        }
         if (!make_map(&maps->new_v, a.kv_fp8 ? a.new_v_codes : a.new_v, 3, dims, str, box)) return false;
     }
     if (a.kv_fp8) {
@@ -308,10 +321,11 @@ inline bool cached_tile_maps(TileMapCache* cache, const KernelArgs& a, int64_t t
                              int block_n, TileMaps* maps) {
     static_assert(sizeof(TileMaps) == 5 * 128, "five tensor maps");
     if (!cache) return build_tile_maps(a, token_rows, D, G, q_tile_tokens, block_n, maps);
-    const void* nk = a.kv_fp8 ? (const void*)a.new_k_codes : (const void*)a.new_k;
+    const void* nk = a.q_fp8 ? (const void*)a.new_k_codes8 : a.kv_fp8 ? (const void*)a.new_k_codes : (const void*)a.new_k;
+    const void* qp = a.q_fp8 ? (const void*)a.q_codes : (const void*)a.q;
     const void* nv = a.kv_fp8 ? (const void*)a.new_v_codes : (const void*)a.new_v;
     for (auto& e : cache->entries) {
-        if (e.valid && e.q == a.q && e.out == a.out && e.new_k == nk && e.new_v == nv && e.kv_cache == a.kv_cache &&
+        if (e.valid && e.q == qp && e.q_fp8 == a.q_fp8 && e.out == a.out && e.new_k == nk && e.new_v == nv && e.kv_cache == a.kv_cache &&
             e.token_rows == token_rows && e.h_q == a.h_q && e.h_kv == a.h_kv && e.head_dim == D && e.page_size == a.page_size &&
             e.num_pages == a.num_pages && e.kv_fp8 == a.kv_fp8 && e.block_n == block_n && e.q_tile_tokens == q_tile_tokens) {
             memcpy(maps, e.maps, sizeof(TileMaps));
@@ -322,7 +336,7 @@ inline bool cached_tile_maps(TileMapCache* cache, const KernelArgs& a, int64_t t
     auto& e = cache->entries[cache->next];
     cache->next = (cache->next + 1) % TileMapCache::kEntries;
     e.valid = true;
-    e.q = a.q, e.out = a.out, e.new_k = nk, e.new_v = nv, e.kv_cache = a.kv_cache;
+    e.q = qp, e.q_fp8 = a.q_fp8, e.out = a.out, e.new_k = nk, e.new_v = nv, e.kv_cache = a.kv_cache;
     e.token_rows = token_rows;
     e.h_q = a.h_q, e.h_kv = a.h_kv, e.head_dim = D, e.page_size = a.page_size, e.num_pages = a.num_pages, e.kv_fp8 = a.kv_fp8;
     e.block_n = block_n, e.q_tile_tokens = q_tile_tokens;

@@ -71,9 +71,15 @@ struct TileCfg {
 enum { BAR_Q = 0, BAR_KFULL = 2, BAR_KEMPTY = 4, BAR_VFULL = 6, BAR_VEMPTY = 8, BAR_SFULL = 10, BAR_PREADY = 12, BAR_ODONE = 14, BAR_UPD = 16, BAR_EPI = 18, BAR_KCONV = 20, BAR_VCONV = 22, BAR_NEXT = 24, BAR_COUNT = 25 };
 
 
-template <int D, int G, bool FP8>
+// QF8 (FP8 cache with a per-tensor scale for Q as well, d_k = 128): the score product runs as
+// tcgen05.mma kind::f8f6f4 straight on code bytes - the query tile arrives as E4M3 codes (16 KB
+// instead of 32), a key block as the raw code rows of the cache (or of the scratch copy of the
+// batch's own K codes), 32 elements of d_k per instruction at twice the bf16 rate - so no key is
+// expanded to bf16 any more; V keeps its bf16 expansion, P being bf16.
+template <int D, int G, bool FP8, bool QF8>
 __global__ void __launch_bounds__(kTileThreads, 1)
 rpa_tile_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
+    static_assert(!QF8 || (FP8 && D == 128), "the FP8 score product is built for an FP8 cache and d_k = 128");
     using C = TileCfg<D>;
     constexpr int TQ = 128 / G;  // tokens per query tile
     extern __shared__ uint8_t smem_raw[];
@@ -179,11 +185,16 @@ rpa_tile_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
                 mbar_arrive(q_bar);
                 return;
             }
-            mbar_arrive_expect_tx(q_bar, n_tiles * C::TILE_BYTES);
-            for (int x = 0; x < n_tiles; ++x)
+            mbar_arrive_expect_tx(q_bar, n_tiles * (QF8 ? C::BLK_BYTES : C::TILE_BYTES));
+            for (int x = 0; x < n_tiles; ++x) {
+                if constexpr (QF8) {  // 128 rows of 128 code bytes
+                    tma_load_3d(region + x * C::TILE_BYTES, &maps.q, 0, head * G, tok_row + x * TQ, q_bar);
+                } else {
 #pragma unroll
-                for (int b = 0; b < C::NBLK; ++b)
-                    tma_load_3d(region + x * C::TILE_BYTES + b * C::BLK_BYTES, &maps.q, b * 64, head * G, tok_row + x * TQ, q_bar);
+                    for (int b = 0; b < C::NBLK; ++b)
+                        tma_load_3d(region + x * C::TILE_BYTES + b * C::BLK_BYTES, &maps.q, b * 64, head * G, tok_row + x * TQ, q_bar);
+                }
+            }
         };
         if (lane == 0) {
             prefetch_tmap(&maps.q);
@@ -227,7 +238,7 @@ rpa_tile_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
                     if (lane == 0) mbar_arrive(bar(full));
                     continue;
                 }
-                if (lane == 0) mbar_arrive_expect_tx(bar(full), bytes);
+                if (lane == 0) mbar_arrive_expect_tx(bar(full), (QF8 && !ctx && kv == 0) ? (uint32_t)C::BLK_BYTES : bytes);
                 __syncwarp();
                 if (ctx) {
                     if (sub_valid) {
@@ -243,9 +254,13 @@ rpa_tile_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
                         }
                     }
                 } else if (lane == 0) {
+                    if (QF8 && kv == 0) {  // the batch's own K codes, where a context block's raw rows land
+                        tma_load_3d(dst + C::BLK_BYTES, &maps.new_k, 0, h, new_row0, bar(full));
+                    } else {
 #pragma unroll
-                    for (int b = 0; b < C::NBLK; ++b)
-                        tma_load_3d(dst + b * C::BLK_BYTES, kv ? &maps.new_v : &maps.new_k, b * 64, h, new_row0, bar(full));
+                        for (int b = 0; b < C::NBLK; ++b)
+                            tma_load_3d(dst + b * C::BLK_BYTES, kv ? &maps.new_v : &maps.new_k, b * 64, h, new_row0, bar(full));
+                    }
                 }
             }
         }
@@ -267,7 +282,7 @@ rpa_tile_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
         }
       } else if (warp == 1) {
         // ================================ MMA issuer ================================
-        constexpr uint32_t idesc_qk = instr_desc_bf16(128, kBlockN, 0, 0);
+        constexpr uint32_t idesc_qk = QF8 ? instr_desc_e4m3(128, kBlockN, 0, 0) : instr_desc_bf16(128, kBlockN, 0, 0);
         constexpr uint32_t idesc_pv = instr_desc_bf16(128, D, 0, 1);
         // Descriptors differ only in their 14-bit start-address field, so each product is issued
         // with one 32-bit add per operand: the issuing thread must not become the bottleneck.  For
@@ -278,16 +293,23 @@ rpa_tile_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
         // that the lanes are together at each election.
         constexpr uint32_t desc_hi = smem_desc_sw128_hi(1024);
         const uint32_t q_lo[2] = {smem_desc_sw128_lo(smem_base + q_off, 16), smem_desc_sw128_lo(smem_base + q_off + C::TILE_BYTES, 16)};
-        const uint32_t k_lo = smem_desc_sw128_lo(smem_base + k_off, 16);
+        // (FP8 scores: the key operand is the raw code rows, which sit in the second half of a K stage)
+        const uint32_t k_lo = smem_desc_sw128_lo(smem_base + k_off + (QF8 ? C::BLK_BYTES : 0), 16);
         const uint32_t v_lo = smem_desc_sw128_lo(smem_base + C::OFF_V, C::BLK_BYTES);
         const bool no_compute = a.ablation & kAblateCompute;  // bench switch: commits without products
         auto issue_qk = [&](int x, int st) {  // S_x = Q_x K^T over d_k in steps of 16
             if (no_compute) return;
             const uint32_t kl = k_lo + st * (C::TILE_BYTES >> 4);
+            if constexpr (QF8) {
 #pragma unroll
-            for (int ks = 0; ks < D / 16; ++ks) {
-                const uint32_t off = ((ks / 4) * C::BLK_BYTES + (ks % 4) * 32) >> 4;
-                umma_ss(tm_s[x], make_desc(q_lo[x] + off, desc_hi), make_desc(kl + off, desc_hi), idesc_qk, ks > 0);
+                for (int ks = 0; ks < D / 32; ++ks)  // 32 code bytes of every row per product
+                    umma_ss_f8(tm_s[x], make_desc(q_lo[x] + ks * 2, desc_hi), make_desc(kl + ks * 2, desc_hi), idesc_qk, ks > 0);
+            } else {
+#pragma unroll
+                for (int ks = 0; ks < D / 16; ++ks) {
+                    const uint32_t off = ((ks / 4) * C::BLK_BYTES + (ks % 4) * 32) >> 4;
+                    umma_ss(tm_s[x], make_desc(q_lo[x] + off, desc_hi), make_desc(kl + off, desc_hi), idesc_qk, ks > 0);
+                }
             }
         };
         auto issue_pv = [&](int x, int st, bool first) {  // O_x (+)= P_x V over 128 positions in steps of 16
@@ -299,7 +321,7 @@ rpa_tile_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
         };
         // barrier that says block j's K (or V) operand is in place: with an FP8 cache a context
         // block is ready once the converter warps have expanded it, not when its bytes land
-        auto k_ready = [&](int j) { return bar((FP8 && j < n_ctx_blocks ? BAR_KCONV : BAR_KFULL) + (j & 1)); };
+        auto k_ready = [&](int j) { return bar((FP8 && !QF8 && j < n_ctx_blocks ? BAR_KCONV : BAR_KFULL) + (j & 1)); };
         auto v_ready = [&](int j) { return bar((FP8 && j < n_ctx_blocks ? BAR_VCONV : BAR_VFULL) + (j & 1)); };
         const bool two_tiles = it.n_tok > TQ;  // a short item (at most TQ tokens) runs tile A only
         const bool split = !two_tiles && n_blocks >= 2;  // ... with its key blocks dealt to both accumulators
@@ -311,10 +333,16 @@ rpa_tile_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
             auto issue_qk_a = [&](int x, int st) {
                 if (no_compute) return;
                 const uint32_t kl = k_lo + st * (C::TILE_BYTES >> 4);
+                if constexpr (QF8) {
 #pragma unroll
-                for (int ks = 0; ks < D / 16; ++ks) {
-                    const uint32_t off = ((ks / 4) * C::BLK_BYTES + (ks % 4) * 32) >> 4;
-                    umma_ss(tm_s[x], make_desc(q_lo[0] + off, desc_hi), make_desc(kl + off, desc_hi), idesc_qk, ks > 0);
+                    for (int ks = 0; ks < D / 32; ++ks)
+                        umma_ss_f8(tm_s[x], make_desc(q_lo[0] + ks * 2, desc_hi), make_desc(kl + ks * 2, desc_hi), idesc_qk, ks > 0);
+                } else {
+#pragma unroll
+                    for (int ks = 0; ks < D / 16; ++ks) {
+                        const uint32_t off = ((ks / 4) * C::BLK_BYTES + (ks % 4) * 32) >> 4;
+                        umma_ss(tm_s[x], make_desc(q_lo[0] + off, desc_hi), make_desc(kl + off, desc_hi), idesc_qk, ks > 0);
+                    }
                 }
             };
             if (ok) {
@@ -491,7 +519,7 @@ rpa_tile_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
                 const int st = j & 1, ph = (j >> 1) & 1;
                 const int rows = min(kBlockN, (min(kBlockN, c - j * kBlockN) + box_rows - 1) / box_rows * box_rows);
 #pragma unroll
-                for (int kv = 0; kv < 2; ++kv) {
+                for (int kv = QF8 ? 1 : 0; kv < 2; ++kv) {  // (FP8 scores: the keys are used as they are)
                     okc = okc && mbar_wait(bar((kv ? BAR_VFULL : BAR_KFULL) + st), ph, abort_flag, a.status, 0x50 + kv);
                     if (!okc) break;
                     uint8_t* stage = smem + (kv ? (uint32_t)C::OFF_V : k_off) + st * C::TILE_BYTES;
@@ -792,19 +820,31 @@ rpa_tile_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
 
 template <int D, int G, bool FP8>
 cudaError_t launch_tile(const KernelArgs& a, int64_t token_rows, TileMapCache* cache, cudaStream_t stream) {
+    constexpr bool kCanQF8 = FP8 && D == 128;
+    if (a.q_fp8 && !kCanQF8) return cudaErrorInvalidValue;
     TileMaps maps;
     if (!cached_tile_maps(cache, a, token_rows, D, G, 128 / G, kBlockN, &maps)) return cudaErrorInvalidValue;
     if (FP8) {
         if (cudaError_t e = launch_quantise_new<D>(a, stream); e != cudaSuccess) return e;
     }
     const int grid = a.dev_counts ? a.num_tile_ctas : a.num_tile_ctas > 0 && a.num_tile_ctas < a.num_tile_items ? a.num_tile_ctas : a.num_tile_items;
-    rpa_tile_kernel<D, G, FP8><<<grid, kTileThreads, TileCfg<D>::SMEM, stream>>>(a, maps);
+    if constexpr (kCanQF8) {
+        if (a.q_fp8) {
+            rpa_tile_kernel<D, G, true, true><<<grid, kTileThreads, TileCfg<D>::SMEM, stream>>>(a, maps);
+            return cudaGetLastError();
+        }
+    }
+    rpa_tile_kernel<D, G, FP8, false><<<grid, kTileThreads, TileCfg<D>::SMEM, stream>>>(a, maps);
     return cudaGetLastError();
 }
 
 template <int D, int G, bool FP8>
 cudaError_t prepare_tile() {
-    return cudaFuncSetAttribute(rpa_tile_kernel<D, G, FP8>, cudaFuncAttributeMaxDynamicSharedMemorySize, TileCfg<D>::SMEM);
+    if constexpr (FP8 && D == 128) {
+        cudaError_t e = cudaFuncSetAttribute(rpa_tile_kernel<D, G, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, TileCfg<D>::SMEM);
+        if (e != cudaSuccess) return e;
+    }
+    return cudaFuncSetAttribute(rpa_tile_kernel<D, G, FP8, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, TileCfg<D>::SMEM);
 }
 
 #define RPA_TILE_DISPATCH(D_, G_, F8_, FN, ...)                         \
