@@ -208,61 +208,80 @@ rpa_tile_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
         const int box_rows = page_box_rows(ps, kBlockN);
         const int sub_blocks = kBlockN / box_rows;
         bool ok = true;
-        for (int j = 0; j < n_blocks && ok; ++j) {
-            const bool ctx = j < n_ctx_blocks;
-            // sources of this block
-            int page = 0, slot0 = 0;
-            bool sub_valid = false;
-            int n_sub_valid = 0;
-            if (ctx) {
+        // where a block comes from: for a context block, this lane's page and first slot
+        struct Src {
+            int page, slot0, n_sub_valid;
+            bool sub_valid;
+        };
+        auto source_of = [&](int j) {
+            Src s{0, 0, 0, false};
+            if (j < n_ctx_blocks) {
                 const int pos = j * kBlockN + lane * box_rows;
-                sub_valid = lane < sub_blocks && pos < c;
-                if (sub_valid) {
-                    page = debug_read_page(a, pt_row[pos / ps]);
-                    slot0 = pos % ps;
+                s.sub_valid = lane < sub_blocks && pos < c;
+                if (s.sub_valid) {
+                    s.page = debug_read_page(a, pt_row[pos / ps]);
+                    s.slot0 = pos % ps;
                 }
-                n_sub_valid = __popc(__ballot_sync(0xffffffffu, sub_valid));
+                s.n_sub_valid = __popc(__ballot_sync(0xffffffffu, s.sub_valid));
             }
+            return s;
+        };
+        // fills stage j & 1 of the K (kv = 0) or V (kv = 1) ring with block j
+        auto fill = [&](int j, int kv, const Src& src) -> bool {
+            const bool ctx = j < n_ctx_blocks;
             const int new_row0 = cu + (j - n_ctx_blocks) * kBlockN;
-            const uint32_t bytes = ctx ? (uint32_t)n_sub_valid * box_rows * D * (FP8 ? 1 : 2) : (uint32_t)C::TILE_BYTES;
-#pragma unroll
-            for (int kv = 0; kv < 2; ++kv) {  // 0: K stage, 1: V stage
-                const int st = j & 1;
-                if (!debug_stage_ok(a, st, C::KS)) break;
-                const int full = (kv ? BAR_VFULL : BAR_KFULL) + st, empty = (kv ? BAR_VEMPTY : BAR_KEMPTY) + st;
-                if (j >= 2) ok = ok && mbar_wait(bar(empty), ((j >> 1) - 1) & 1, abort_flag, a.status, 0x10 + kv);
-                ok = __all_sync(0xffffffffu, ok);
-                if (!ok) break;
-                const uint32_t dst = (kv ? smem_base + C::OFF_V : k_region) + st * C::TILE_BYTES;
-                if (a.ablation & kAblateLoads) {
-                    if (lane == 0) mbar_arrive(bar(full));
-                    continue;
-                }
-                if (lane == 0) mbar_arrive_expect_tx(bar(full), (QF8 && !ctx && kv == 0) ? (uint32_t)C::BLK_BYTES : bytes);
-                __syncwarp();
-                if (ctx) {
-                    if (sub_valid) {
-                        if constexpr (FP8) {
-                            // raw FP8 rows (d_k bytes each) land in the upper half of the stage
-                            tma_load_4d(dst + C::BLK_BYTES + lane * box_rows * 128, &maps.cache, 0, 2 * h + kv, slot0, page,
-                                        bar(full));
-                        } else {
-#pragma unroll
-                            for (int b = 0; b < C::NBLK; ++b)
-                                tma_load_4d(dst + b * C::BLK_BYTES + lane * box_rows * 128, &maps.cache, b * 64, 2 * h + kv, slot0,
-                                            page, bar(full));
-                        }
-                    }
-                } else if (lane == 0) {
-                    if (QF8 && kv == 0) {  // the batch's own K codes, where a context block's raw rows land
-                        tma_load_3d(dst + C::BLK_BYTES, &maps.new_k, 0, h, new_row0, bar(full));
+            const uint32_t bytes = ctx ? (uint32_t)src.n_sub_valid * box_rows * D * (FP8 ? 1 : 2) : (uint32_t)C::TILE_BYTES;
+            const int st = j & 1;
+            if (!debug_stage_ok(a, st, C::KS)) return false;
+            const int full = (kv ? BAR_VFULL : BAR_KFULL) + st, empty = (kv ? BAR_VEMPTY : BAR_KEMPTY) + st;
+            bool good = true;
+            if (j >= 2) good = mbar_wait(bar(empty), ((j >> 1) - 1) & 1, abort_flag, a.status, 0x10 + kv);
+            good = __all_sync(0xffffffffu, good);
+            if (!good) return false;
+            const uint32_t dst = (kv ? smem_base + C::OFF_V : k_region) + st * C::TILE_BYTES;
+            if (a.ablation & kAblateLoads) {
+                if (lane == 0) mbar_arrive(bar(full));
+                return true;
+            }
+            if (lane == 0) mbar_arrive_expect_tx(bar(full), (QF8 && !ctx && kv == 0) ? (uint32_t)C::BLK_BYTES : bytes);
+            __syncwarp();
+            if (ctx) {
+                if (src.sub_valid) {
+                    if constexpr (FP8) {
+                        // raw FP8 rows (d_k bytes each) land in the upper half of the stage
+                        tma_load_4d(dst + C::BLK_BYTES + lane * box_rows * 128, &maps.cache, 0, 2 * h + kv, src.slot0, src.page,
+                                    bar(full));
                     } else {
 #pragma unroll
                         for (int b = 0; b < C::NBLK; ++b)
-                            tma_load_3d(dst + b * C::BLK_BYTES, kv ? &maps.new_v : &maps.new_k, b * 64, h, new_row0, bar(full));
+                            tma_load_4d(dst + b * C::BLK_BYTES + lane * box_rows * 128, &maps.cache, b * 64, 2 * h + kv, src.slot0,
+                                        src.page, bar(full));
                     }
                 }
+            } else if (lane == 0) {
+                if (QF8 && kv == 0) {  // the batch's own K codes, where a context block's raw rows land
+                    tma_load_3d(dst + C::BLK_BYTES, &maps.new_k, 0, h, new_row0, bar(full));
+                } else {
+#pragma unroll
+                    for (int b = 0; b < C::NBLK; ++b)
+                        tma_load_3d(dst + b * C::BLK_BYTES, kv ? &maps.new_v : &maps.new_k, b * 64, h, new_row0, bar(full));
+                }
             }
+            return true;
+        };
+        // The keys run one block ahead of the values: K(j+1) goes out before V(j).  A V stage is held
+        // much longer than a K stage (until the PV product of its block, i.e. through that block's whole
+        // softmax), and with the loads in block order the wait for a free V stage also held back the
+        // next block's keys, whose stage had long been free.
+        Src prev{0, 0, 0, false};
+        for (int t = 0; t <= n_blocks && ok; ++t) {
+            Src cur{0, 0, 0, false};
+            if (t < n_blocks) {
+                cur = source_of(t);
+                ok = fill(t, 0, cur);
+            }
+            if (ok && t >= 1) ok = fill(t - 1, 1, prev);
+            prev = cur;
         }
         // the next item's query tiles, into this item's K ring once its last score product has read it
         if (ok) ok = mbar_wait(bar(BAR_NEXT), 0, abort_flag, a.status, 0x12);
