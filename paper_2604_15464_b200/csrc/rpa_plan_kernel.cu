@@ -35,7 +35,7 @@ __device__ __forceinline__ int64_t round_up64(int64_t a, int64_t b) { return cei
 __device__ __forceinline__ bool dev_routed_to_tile(const DevPlanArgs& p, int64_t q_r, int64_t L_r) {
     if (p.tile_min_q <= 0) return false;
     if (q_r >= p.tile_min_q) return true;
-    return p.tile_long_q > 0 && q_r >= p.tile_long_q && L_r >= p.tile_long_kv && p.page_size >= 64;
+    return p.tile_long_q > 0 && q_r >= p.tile_long_q && L_r >= p.tile_long_kv && p.page_size >= kTileLongPage;
 }
 
 // The split of one row unit (up to tpi tokens of one sequence starting at t0), as the host planner

@@ -38,7 +38,7 @@ void sort_longest_first(Plan& plan) {
 inline bool routed_to_tile(const rpa_config_t& cfg, const PlanPolicy& policy, int64_t q_r, int64_t L_r) {
     if (policy.tile_min_q <= 0) return false;
     if (q_r >= policy.tile_min_q) return true;
-    return policy.tile_long_q > 0 && q_r >= policy.tile_long_q && L_r >= kTileLongKv && cfg.page_size >= 64;
+    return policy.tile_long_q > 0 && q_r >= policy.tile_long_q && L_r >= kTileLongKv && cfg.page_size >= kTileLongPage;
 }
 
 }  // namespace

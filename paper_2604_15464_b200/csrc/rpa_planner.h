@@ -20,7 +20,7 @@ struct PlanPolicy {
     int kv_chunk_override = 0;  // > 0: split-KV chunk length in tokens (multiple of kKvTile)
     int tile_min_q = 0;         // sequences with q_len >= this go to the tile kernel; 0 = none
     int tile_long_q = 0;        // > 0: sequences with q_len >= this also go to the tile kernel when their
-                                // context is long (>= kTileLongKv tokens) and pages are large (>= 64 slots)
+                                // context is long (>= kTileLongKv tokens) and pages are not small (>= kTileLongPage slots)
     int tile_tokens = 0;        // query tokens per tile item
     bool pack_short = false;    // pack runs of short sequences without context into one tile item
     int max_row_items = 0;      // capacities of the device lists

@@ -15,6 +15,10 @@ constexpr int kRefineFactors[8] = {8, 10, 12, 14, 18, 20, 24, 32};
 constexpr int kItemFixedKeys = 192;       // measured: about 4 us per item
 constexpr int kSplitItemFixedKeys = 400;  // an item of a split sequence also writes its partial, and one of them merges the group
 constexpr long long kTileGlobalOrderBytes = 72ll << 20;  // K/V of the tile-routed sequences up to which tile items are ordered across heads
+// Sequences with a few query rows more than one row item holds go to the tile kernel when their context
+// is long and their pages have at least this many slots (with 16-slot pages the tile kernel's per-page
+// TMA boxes are too small for it to beat two row items; from 32 slots on it streams at 6.1 TB/s against 5.0)
+constexpr int kTileLongPage = 32;
 constexpr int kQTile = 128;       // query rows per tile-kernel item (tcgen05 M)
 
 constexpr int kFlagWriteKv = 1;   // this item copies its new tokens' K/V rows into the cache
