@@ -343,7 +343,7 @@ rpa_status_t rpa_set_kv_chunk(rpa_handle_t* h, int32_t tokens);
  * the row kernel, and nothing else decides: an explicit threshold switches off the packing of short
  * sequences and the extra rule for small queries on long contexts.  0 restores the default rules
  * (tile kernel from more than two row items' worth of query rows, q*h_g > 32; from more than one
- * with at least 1024 keys on pages of 64 slots or more; runs of short sequences without context
+ * with at least 1024 keys on pages of 32 slots or more; runs of short sequences without context
  * packed into shared tile items); a value above max_num_tokens keeps everything on the row kernel.
  * Invalidates the current plan.  Meant for tests and tuning. */
 rpa_status_t rpa_set_tile_min_q(rpa_handle_t* h, int32_t tokens);
