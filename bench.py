@@ -467,6 +467,10 @@ def run_leg(workload, args, rank, world, local, dist, peaks):
         cpu_baseline = cpu_baseline_of(meta, batch, unit, args.cpu_budget)
 
     rapi.close()
+    clock_summary = clocks.summary()
+    # the same figure per GHz of the SM clock sampled during the timed blocks: under the power cap the
+    # clock moves from run to run, and this tells a slower kernel from a slower clock
+    per_ghz = value / (clock_summary["sm_mhz"] / 1e3) if clock_summary.get("sm_mhz") else None
     launches_per_step = device_plan_launches(meta) if args.plan == "device" else info["gpu_launches"]
     return {
         "metric": metric, "value": value, "unit": unit, "n_gpus": world, "steps": args.steps,
@@ -486,7 +490,8 @@ def run_leg(workload, args, rank, world, local, dist, peaks):
         "timing": {"blocks": len(block_ms), "steps_per_block": args.steps, "gpu_seconds_timed": busy_ms * 1e-3,
                    "block_ms_median": median(block_ms), "block_ms_min": min(block_ms), "block_ms_max": max(block_ms),
                    "per_kernel_events_in_timed_blocks": False},
-        "clocks": clocks.summary(),
+        "clocks": clock_summary,
+        "value_per_sm_ghz": per_ghz,
         "roofline": roofline,
         "roofline_other_kernels": other,
         "e2e": e2e,
