@@ -16,11 +16,12 @@ BF16_BYTES = 2
 def algorithmic_bytes(q_lens: Sequence[int], kv_lens: Sequence[int], num_q_heads: int, num_kv_heads: int,
                       head_dim: int, data_bytes: int = BF16_BYTES) -> int:
     """Bytes the method must move: every K/V token of the context read once (cached or new), every
-    new token written to the cache once, Q read and the output written.  With n equal requests of
-    q_len 1 this is the numerator of the paper's decode throughput (Section 4.1.1)."""
+    new token written to the cache once, Q read and the output written.  A request without new tokens
+    moves nothing (nobody attends to its context in this call).  With n equal requests of q_len 1 this
+    is the numerator of the paper's decode throughput (Section 4.1.1)."""
     token_bytes = 2 * num_kv_heads * head_dim * data_bytes
     qo_bytes = 2 * num_q_heads * head_dim * data_bytes
-    return int(sum((int(L) + int(q)) * token_bytes + int(q) * qo_bytes for q, L in zip(q_lens, kv_lens)))
+    return int(sum((int(L) + int(q)) * token_bytes + int(q) * qo_bytes for q, L in zip(q_lens, kv_lens) if int(q) > 0))
 
 
 def attention_flops(q_lens: Sequence[int], kv_lens: Sequence[int], num_q_heads: int, head_dim: int,
