@@ -67,6 +67,36 @@ def test_device_lists_equal_host_lists():
     _lists_match(nc, kv_chunk=64)
 
 
+@pytest.mark.parametrize("seed", range(16))
+def test_device_lists_equal_host_lists_on_random_batches(seed):
+    """The two planners are separate code (C++ on the host, one CUDA block on the device): seeded
+    random batches over head shapes, page sizes, masks and lengths must give the same lists."""
+    rng = np.random.default_rng(6000 + seed)
+    d = int(rng.choice([64, 128, 256]))
+    h_kv = int(rng.choice([1, 2, 8]))
+    h_g = int(rng.choice([1, 2, 4, 8, 16]))
+    ps = int(rng.choice([16, 32, 48, 64, 128, 256]))
+    n = int(rng.integers(1, 40))
+    q_lens, kv_lens = [], []
+    for _ in range(n):
+        kind = int(rng.integers(0, 5))
+        if kind == 0:
+            q, ctx = 1, int(rng.integers(0, 12000))
+        elif kind == 1:
+            q, ctx = int(rng.integers(2, 40)), int(rng.integers(0, 3000))
+        elif kind == 2:
+            q, ctx = int(rng.integers(40, 500)), int(rng.integers(0, 2000))
+        elif kind == 3:
+            q, ctx = int(rng.integers(1, 40)), 0
+        else:
+            q, ctx = 0, int(rng.integers(0, 50))
+        q_lens.append(q)
+        kv_lens.append(q + ctx)
+    meta = wl.build_meta(f"dpr{seed}", q_lens, kv_lens, num_q_heads=h_kv * h_g, num_kv_heads=h_kv, head_dim=d, page_size=ps,
+                         causal=bool(rng.integers(0, 4) > 0), seed=seed, token_capacity=sum(q_lens) + 4)
+    _lists_match(meta)
+
+
 @pytest.mark.parametrize("cfg", [1, 4])
 def test_device_planned_step_matches_oracle(cfg):
     batch = wl.materialize(wl.workload_meta(cfg), _dev(), canaries=(cfg == 1))
