@@ -102,3 +102,27 @@ def test_random_batches_on_unaligned_page_sizes(seed):
     tile_min_q = [None, 1, 8][seed % 3]
     batch = wl.materialize(meta, torch.device("cuda", 0), canaries=bool(seed % 2))
     hz.full_parity(batch, tile_min_q=tile_min_q, device_plan=(tile_min_q is None and seed % 4 == 0))
+
+
+@pytest.mark.parametrize("seed", range(10))
+def test_random_batches_with_quantised_q_and_the_bounds_checked_build(seed):
+    """FP8 caches with a scale for Q as well (FP8 score products on the d_k = 128 tile path), host- and
+    device-planned, every other batch through the bounds-checked build of the library, which must
+    report nothing on good input."""
+    from paper_2604_15464_b200 import binding
+
+    rng = np.random.default_rng(3000 + seed)
+    case = _random_case(rng, n_max=10, kinds=6)
+    q_lens, kv_lens = case.pop("q_lens"), case.pop("kv_lens")
+    if rng.integers(0, 2):
+        q = int(rng.integers(2, 200))
+        q_lens.append(q)
+        kv_lens.append(q + int(rng.integers(500, 3000)))
+    meta = wl.build_meta(f"randq{seed}", q_lens, kv_lens, seed=700 + seed, token_capacity=sum(q_lens) + 2, kv_fp8=True,
+                         k_scale=0.03, v_scale=0.025, q_scale=float(rng.choice([0.02, 0.03125, 0.05])), **case)
+    lib = build.build(debug=True) if seed % 2 else None
+    rapi = binding.Rpa.for_meta(meta, library_path=lib)
+    batch = wl.materialize(meta, torch.device("cuda", 0), canaries=bool(seed % 3 == 0))
+    hz.full_parity(batch, rapi=rapi, device_plan=bool(seed % 4 == 1))
+    assert rapi.rpa_poll_status() == 0
+    rapi.close()
