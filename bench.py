@@ -346,6 +346,8 @@ def run_leg(workload, args, rank, world, local, dist, peaks):
         rapi.rpa_set_kv_chunk(args.kv_chunk)
     if args.ablate:
         rapi.rpa_set_ablation(args.ablate)
+    if args.tile_pair is not None:
+        rapi.rpa_set_tile_pair(args.tile_pair)
     out = torch.zeros_like(batch.q)
     stream = torch.cuda.current_stream()
     sh = stream.cuda_stream
@@ -567,6 +569,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--plan-only", action="store_true", help="no device: plan the headline batch on every rank and print the launch's shape")
     ap.add_argument("--kv-chunk", type=int, default=0)
+    ap.add_argument("--tile-pair", type=int, default=None, choices=[0, 1], help="rpa_set_tile_pair: tile items on the CTA-pair kernel (1) or the two-tile kernel (0)")
     ap.add_argument("--ablate", type=int, default=0, help="rpa_set_ablation mask (1: no cache update, 2: no kernel overlap, 4: no attention arithmetic, 8: no K/V loads)")
     ap.add_argument("--ctx", type=int, default=8192, help="context length of the paper_decode workload")
     ap.add_argument("--seq", type=int, default=8192, help="sequence length of the paper_prefill workload")

@@ -348,6 +348,14 @@ rpa_status_t rpa_set_kv_chunk(rpa_handle_t* h, int32_t tokens);
  * Invalidates the current plan.  Meant for tests and tuning. */
 rpa_status_t rpa_set_tile_min_q(rpa_handle_t* h, int32_t tokens);
 
+/* Tile items of host-made plans on the CTA-pair kernel (mode 1) or on the two-tile kernel (mode 0,
+ * the default).  The pair kernel runs Algorithm 1's products for four query tiles at a time on two
+ * neighbouring SMs that share every key block (each stages half of it); an item then covers twice
+ * the tokens.  bf16 cache and d_k = 128 only (RPA_ERR_UNSUPPORTED otherwise); plans made on the
+ * device keep the two-tile kernel.  Invalidates the current plan.  Results are the same function of
+ * the inputs either way (same tolerance against the definition, cache bytes identical). */
+rpa_status_t rpa_set_tile_pair(rpa_handle_t* h, int32_t mode);
+
 const char* rpa_status_string(rpa_status_t s);
 
 /* Text of the last CUDA error seen by this handle ("" if none). */

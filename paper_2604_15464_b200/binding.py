@@ -25,7 +25,7 @@ ABLATE_OVERLAP = 2
 EXPORTS = ["rpa_create", "rpa_destroy", "rpa_plan", "rpa_forward", "rpa_forward_host", "rpa_forward_host_submit",
            "rpa_forward_host_wait", "rpa_plan_info",
            "rpa_plan_dump", "rpa_poll_status", "rpa_set_ablation", "rpa_set_kv_chunk", "rpa_set_kernel_timing",
-           "rpa_get_kernel_timing", "rpa_forward_static", "rpa_set_tile_min_q", "rpa_selftest_bounded_wait", "rpa_set_validation", "rpa_plan_device", "rpa_plan_device_dump",
+           "rpa_get_kernel_timing", "rpa_forward_static", "rpa_set_tile_min_q", "rpa_set_tile_pair", "rpa_selftest_bounded_wait", "rpa_set_validation", "rpa_plan_device", "rpa_plan_device_dump",
            "rpa_status_string",
            "rpa_last_cuda_error"]
 
@@ -84,6 +84,7 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.rpa_set_ablation.argtypes = [vp, ctypes.c_uint32]
     lib.rpa_set_kv_chunk.argtypes = [vp, i32]
     lib.rpa_set_tile_min_q.argtypes = [vp, i32]
+    lib.rpa_set_tile_pair.argtypes = [vp, i32]
     lib.rpa_selftest_bounded_wait.argtypes = [vp, vp]
     lib.rpa_set_validation.argtypes = [vp, i32]
     lib.rpa_plan_device.argtypes = [vp, vp, vp, i32, vp]
@@ -283,6 +284,9 @@ class Rpa:
 
     def rpa_set_tile_min_q(self, tokens: int) -> None:
         self._check(self._lib.rpa_set_tile_min_q(self._h, tokens), "rpa_set_tile_min_q")
+
+    def rpa_set_tile_pair(self, mode: int) -> None:
+        self._check(self._lib.rpa_set_tile_pair(self._h, mode), "rpa_set_tile_pair")
 
     def rpa_set_kernel_timing(self, enable: bool) -> None:
         self._check(self._lib.rpa_set_kernel_timing(self._h, 1 if enable else 0), "rpa_set_kernel_timing")

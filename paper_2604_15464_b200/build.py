@@ -11,7 +11,7 @@ LIB = os.path.join(PKG, "librpa_b200.so")
 # the bounds-checked build (-DRPA_DEBUG): every page id, token row and ring stage is checked before
 # the access and the first violation is recorded in the device status word
 LIB_DEBUG = os.path.join(PKG, "librpa_b200_debug.so")
-SOURCES = ["rpa_api.cu", "rpa_row_kernel.cu", "rpa_row_kernel_fp8.cu", "rpa_tile_kernel.cu", "rpa_tile1_kernel.cu", "rpa_static.cu", "rpa_plan_kernel.cu", "rpa_planner.cc"]
+SOURCES = ["rpa_api.cu", "rpa_row_kernel.cu", "rpa_row_kernel_fp8.cu", "rpa_tile_kernel.cu", "rpa_tile1_kernel.cu", "rpa_tile2_kernel.cu", "rpa_static.cu", "rpa_plan_kernel.cu", "rpa_planner.cc"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "--use_fast_math",
               "-Xcompiler", "-fPIC,-Wall,-Wno-unknown-pragmas", "-Xptxas", "-v"]
 

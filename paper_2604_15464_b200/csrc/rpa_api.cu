@@ -25,6 +25,8 @@ struct rpa_handle {
     Plan plan;
     int planned_num_seqs = -1;
     uint32_t ablation = 0;
+    int tile_pair_mode = 0;  // 0: two-tile kernel only; 1: host-planned steps run their tile items on the CTA-pair kernel
+    bool plan_pair = false;  // the current host-made plan's tile items are pair items
     std::string last_error;
 
     // Device work lists, [row items | tile items | combine groups | kv_lens | cu_q_lens], in a ring of
@@ -255,6 +257,7 @@ rpa_status_t rpa_create(const rpa_config_t* cfg, int device, rpa_handle_t** out)
         if (e == cudaSuccess && cfg->kv_dtype == RPA_KV_FP8_E4M3 && tile_kernel_fp8_supported(cfg->head_dim, h_g))
             e = tile_kernel_prepare(cfg->head_dim, h_g, true);
         if (e == cudaSuccess && tile1_kernel_supported(cfg->head_dim, h_g)) e = tile1_kernel_prepare(cfg->head_dim, h_g);
+        if (e == cudaSuccess && cfg->kv_dtype == RPA_KV_BF16 && tile2_kernel_supported(cfg->head_dim, h_g)) e = tile2_kernel_prepare(h_g);
         if (e != cudaSuccess) {
             delete h;
             return RPA_ERR_CUDA;
@@ -346,8 +349,15 @@ rpa_status_t rpa_plan(rpa_handle_t* h, const int32_t* cu_q_lens_host, const int3
     if (!h) return RPA_ERR_INVALID_ARG;
     h->planned_num_seqs = -1;
     h->device_planned = false;
-    rpa_status_t st = build_plan(h->cfg, h->policy, cu_q_lens_host, kv_lens_host, num_seqs, h->plan);
+    const bool pair = h->tile_pair_mode == 1 && h->policy.tile_min_q > 0;
+    PlanPolicy pol = h->policy;
+    if (pair) {  // pair items: twice the tokens, never packed
+        pol.tile_tokens = tile2_kernel_tokens(h->cfg.num_q_heads / h->cfg.num_kv_heads);
+        pol.pack_short = false;
+    }
+    rpa_status_t st = build_plan(h->cfg, pol, cu_q_lens_host, kv_lens_host, num_seqs, h->plan);
     if (st != RPA_OK) return st;
+    h->plan_pair = pair;
     if (plan_log_enabled()) log_plan(h);
     if (!h->plan_only) {
         st = ensure_device(h);
@@ -678,8 +688,9 @@ rpa_status_t rpa_forward(rpa_handle_t* h, const void* q, const void* new_k, cons
         RPA_CUDA(h, cudaEventRecord(h->ev_fork, s));
         RPA_CUDA(h, cudaStreamWaitEvent(h->aux_stream, h->ev_fork, 0));
         timing_mark(h, 1, h->aux_stream);
-        RPA_CUDA(h, single_tile ? launch_tile1_kernel(a, h->plan.info.num_tokens, &h->tile_maps, h->aux_stream)
-                                : launch_tile_kernel(a, h->plan.info.num_tokens, &h->tile_maps, h->aux_stream));
+        RPA_CUDA(h, h->plan_pair   ? launch_tile2_kernel(a, h->plan.info.num_tokens, &h->tile_maps, h->aux_stream)
+                    : single_tile ? launch_tile1_kernel(a, h->plan.info.num_tokens, &h->tile_maps, h->aux_stream)
+                                  : launch_tile_kernel(a, h->plan.info.num_tokens, &h->tile_maps, h->aux_stream));
         timing_mark(h, 1, h->aux_stream);
         RPA_CUDA(h, cudaEventRecord(h->ev_join, h->aux_stream));
         timing_mark(h, 0, s);
@@ -695,8 +706,9 @@ rpa_status_t rpa_forward(rpa_handle_t* h, const void* q, const void* new_k, cons
         if (a.num_tile_items > 0) {
             a.num_tile_ctas = h->num_sms;  // one after the other: the whole device each, one persistent CTA per SM
             timing_mark(h, 1, s);
-            RPA_CUDA(h, single_tile ? launch_tile1_kernel(a, h->plan.info.num_tokens, &h->tile_maps, s)
-                                    : launch_tile_kernel(a, h->plan.info.num_tokens, &h->tile_maps, s));
+            RPA_CUDA(h, h->plan_pair   ? launch_tile2_kernel(a, h->plan.info.num_tokens, &h->tile_maps, s)
+                        : single_tile ? launch_tile1_kernel(a, h->plan.info.num_tokens, &h->tile_maps, s)
+                                      : launch_tile_kernel(a, h->plan.info.num_tokens, &h->tile_maps, s));
             timing_mark(h, 1, s);
         }
     }
@@ -900,6 +912,16 @@ rpa_status_t rpa_set_tile_min_q(rpa_handle_t* h, int32_t tokens) {
     h->policy.tile_long_q = tokens == 0 ? std::max(2, kRowTileRows / h_g + 1) : 0;  // an explicit threshold is the only rule
     if (!tile_path_available(h->cfg)) h->policy.tile_min_q = h->policy.tile_long_q = 0;
     h->policy.pack_short = tokens == 0 && h->policy.tile_min_q > 0 && !tile1_kernel_supported(h->cfg.head_dim, h_g);
+    h->plan.valid = false;
+    h->planned_num_seqs = -1;
+    return RPA_OK;
+}
+
+rpa_status_t rpa_set_tile_pair(rpa_handle_t* h, int32_t mode) {
+    if (!h || mode < 0 || mode > 1) return RPA_ERR_INVALID_ARG;
+    const int h_g = h->cfg.num_q_heads / h->cfg.num_kv_heads;
+    if (mode && (h->cfg.kv_dtype != RPA_KV_BF16 || !tile2_kernel_supported(h->cfg.head_dim, h_g))) return RPA_ERR_UNSUPPORTED;
+    h->tile_pair_mode = mode;
     h->plan.valid = false;
     h->planned_num_seqs = -1;
     return RPA_OK;

@@ -146,6 +146,13 @@ bool tile1_kernel_supported(int head_dim, int group);
 cudaError_t tile1_kernel_prepare(int head_dim, int group);
 cudaError_t launch_tile1_kernel(const KernelArgs& a, int64_t token_rows, TileMapCache* cache, cudaStream_t stream);
 
+// CTA-pair variant for long prefill (rpa_tile2_kernel.cu): d_k = 128, bf16 cache, host-made plans;
+// an item covers twice the tokens of a two-tile item, half of them per CTA of the pair
+bool tile2_kernel_supported(int head_dim, int group);
+int tile2_kernel_tokens(int group);
+cudaError_t tile2_kernel_prepare(int group);
+cudaError_t launch_tile2_kernel(const KernelArgs& a, int64_t token_rows, TileMapCache* cache, cudaStream_t stream);
+
 // Checks the device copies of the lengths against the plan and every page id a sequence maps
 // against the pool size; a violation sets bit 29 of the status word (low bits: the sequence).
 cudaError_t launch_validate_kernel(const KernelArgs& a, int32_t num_seqs, const int32_t* plan_kv_lens, cudaStream_t stream);

@@ -228,6 +228,112 @@ __device__ __forceinline__ void tc_commit_warp(uint32_t bar) {
         : "memory");
 }
 
+// ---------------------------------------------------------------- CTA pairs (clusters of two)
+// A pair of CTAs on neighbouring SMs runs one tensor product of 256 rows: each CTA holds its 128
+// rows of A and of the accumulator and HALF of the B operand; one thread of the first CTA issues.
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;\n" : "=r"(r));
+    return r;
+}
+// Every thread of both CTAs arrives, then waits: orders memory operations across the pair.  The
+// lanes of a warp arrive together (a warp whose lanes arrived in two groups, one of them late,
+// let the barrier open before the late group had arrived).
+__device__ __forceinline__ void cluster_sync() {
+    __syncwarp();
+    asm volatile("barrier.cluster.arrive.release.aligned;\nbarrier.cluster.wait.acquire.aligned;\n" ::: "memory");
+}
+// address of the same shared-memory location in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;\n" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+// Arrival at a barrier of either CTA.  The plain form orders nothing beyond this CTA: enough where the
+// waiter consumes what the tensor core, the copy engine or TMEM hold (ordered by their own fences).
+// The releasing form publishes the thread's earlier shared-memory writes to the whole pair; it costs
+// about as much as a device-wide fence (1800 cycles measured), so it stays off the per-block path.
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];\n" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster_release(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];\n" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ void st_cluster_u32(uint32_t cluster_addr, uint32_t v) {
+    asm volatile("st.shared::cluster.u32 [%0], %1;\n" ::"r"(cluster_addr), "r"(v) : "memory");
+}
+// the wait of a barrier that the other CTA of the pair may have arrived at
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n"
+        "selp.u32 %0, 1, 0, p;\n"
+        "}\n"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait inside a pair: as mbar_wait, and on expiry the abort flag of the other CTA
+// (`peer_abort`, a cluster address) is raised as well, so that both leave together.  kClusterAcquire:
+// the waiter reads shared memory that a thread of the other CTA wrote before its releasing arrival.
+template <bool kClusterAcquire = false>
+__device__ __forceinline__ bool mbar_wait_pair(uint32_t bar, uint32_t parity, volatile uint32_t* abort, uint32_t peer_abort,
+                                               uint32_t* status, uint32_t code, long long limit = 4000000000LL) {
+    auto done = [&]() { return kClusterAcquire ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity); };
+    if (done()) return true;
+    const long long t0 = clock64();
+    while (!done()) {
+        if (*abort) return false;
+        if (clock64() - t0 > limit) {
+            *abort = 1u;
+            st_cluster_u32(peer_abort, 1u);
+            if (atomicCAS(status, 0u, (1u << 28) | code) != 0u) atomicOr(status, 1u << 28);  // the first wait to give up names itself
+            return false;
+        }
+    }
+    return true;
+}
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t smem_result, uint32_t cols) {  // one warp of EACH CTA
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_result), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish_pair() {
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;\n" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t cols) {
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;\n" ::"r"(taddr), "r"(cols) : "memory");
+}
+// D(tmem of both) (+)= A(smem of each) * B(halves in the smem of each)
+__device__ __forceinline__ void umma_ss_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "setp.ne.b32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n"
+        "}\n" ::"r"(d_tmem),
+        "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void umma_ts_pair(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "setp.ne.b32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], [%1], %2, %3, p;\n"
+        "}\n" ::"r"(d_tmem),
+        "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// All products issued so far by this thread arrive, on completion, on the barrier at this offset in
+// both CTAs of the pair (a signal, not a copy).
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;\n" ::"r"(bar),
+                 "h"((uint16_t)3)
+                 : "memory");
+}
+
 // ---------------------------------------------------------------- TMEM <-> registers
 // 32 lanes x 32 columns of 32 bits: thread t of the warp gets lane (base lane + t), columns c..c+31.
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
