@@ -14,14 +14,24 @@
 // One thread of the pair's first CTA issues all products; completion is signalled to the barriers
 // of both CTAs (tcgen05.commit to both).  Each CTA's producer warp loads its own halves with plain
 // TMA loads into its own shared memory; the second CTA's warp 1 relays "my half has landed" to the
-// first CTA's barriers, and its softmax warps arrive on the first CTA's "P ready" barriers.  Items
-// are drawn by the first CTA and handed to the second through its shared memory.  Algorithm 1's
-// recurrences, the conditional rescale and the fused cache update ("Update U_kv") are those of the
-// two-tile kernel.  Every wait is bounded; a CTA that gives up raises its partner's abort flag too,
-// and neither leaves before both have arrived at the final cluster barrier.
+// first CTA's barriers, and its softmax warps arrive on the first CTA's "P ready" barriers.
 //
-// bf16 cache, d_k = 128, host-made plans, items without packing; everything else runs on the
-// two-tile kernel.
+// Items follow one another without a pause.  Nothing is re-initialised between items and no role
+// waits for another at an item's end: every mbarrier keeps its phase from block to block across
+// items (each role counts the blocks it has seen), the K/V rings run on into the next item's first
+// blocks while the current item's last ones are still being consumed, the query tiles alternate
+// between two buffers, and the score products of the next item's first block are issued right
+// behind the last PV products of the running one - so the output epilogue of an item (TMEM ->
+// shared memory -> bulk store) overlaps the next item's first products instead of idling the
+// tensor pipe.  Items are drawn by one warp of the first CTA from the device-wide counter (the list
+// is sorted heaviest first) a few key blocks before the running item ends, and handed to every
+// role of both CTAs through a two-slot ring in shared memory.
+//
+// Algorithm 1's recurrences, the conditional rescale and the fused cache update ("Update U_kv")
+// are those of the two-tile kernel.  Every wait is bounded; a CTA that gives up raises its
+// partner's abort flag too, and neither leaves before both have arrived at the final cluster
+// barrier.  bf16 cache, d_k = 128, host-made plans, items without packing; everything else runs
+// on the two-tile kernel.
 #include <cuda.h>
 #include <cuda_bf16.h>
 
@@ -39,8 +49,10 @@ namespace {
 constexpr int kBlockN = 128;       // KV positions per block
 constexpr int kHalfN = 64;         // ... of which each CTA of the pair stages this many keys
 constexpr int kPairThreads = 384;  // 12 warps = 3 warpgroups per CTA
+constexpr int kPairWarps = 2 * (kPairThreads / 32);
 constexpr uint32_t kTmemCols = 512;
 constexpr float kRescaleThreshold = 8.f;  // log2 units
+constexpr int kFetchAhead = 3;     // the next item is drawn when the running one has this many key blocks to go
 constexpr int D = 128;
 
 struct PairCfg {
@@ -56,15 +68,18 @@ struct PairCfg {
     static constexpr int OFF_V = OFF_K + KS * K_STAGE;
     static constexpr int OFF_UPD = OFF_V + VS * V_STAGE;  // staging of the fused cache update
     static constexpr int OFF_BAR = OFF_UPD + TileUpdate<D>::STAGE_BYTES;
-    static constexpr int SMEM = OFF_BAR + kTileBarBlockBytes + 1024;
+    static constexpr int OFF_FLAGS = OFF_BAR + 256;  // abort flag, TMEM address, progress
+    static constexpr int OFF_SLOTS = OFF_FLAGS + 64; // two item slots of RAW_INTS ints
+    static constexpr int SMEM = OFF_SLOTS + 2 * RAW_INTS * 4 + 1024;  // + slack for 1024-byte alignment
     static_assert(SMEM <= 232448, "shared memory budget");
 };
 
-// barrier slots (8 bytes each).  Every CTA has all of them at the same offsets; QPEER/KPEER/VPEER
-// and PREADY are used in the first CTA only.
-enum { BAR_Q = 0, BAR_KFULL = 2, BAR_KEMPTY = 4, BAR_VFULL = 6, BAR_VEMPTY = 8, BAR_SFULL = 10, BAR_PREADY = 12, BAR_ODONE = 14,
-       BAR_UPD = 16, BAR_EPI = 18, BAR_NEXT = 20, BAR_QPEER = 21, BAR_KPEER = 22, BAR_VPEER = 24, BAR_COUNT = 26 };
-static_assert(8 * BAR_COUNT + 24 <= 256, "barriers and flags fit in front of the item slots");
+// barrier slots (8 bytes each), two of each kind.  Every CTA has all of them at the same offsets;
+// QPEER/KPEER/VPEER, PREADY and ITEMFREE are used in the first CTA only.
+enum { BAR_Q = 0, BAR_QPEER = 2, BAR_QFREE = 4, BAR_KFULL = 6, BAR_KEMPTY = 8, BAR_VFULL = 10, BAR_VEMPTY = 12, BAR_KPEER = 14,
+       BAR_VPEER = 16, BAR_SFULL = 18, BAR_PREADY = 20, BAR_ODONE = 22, BAR_UPD = 24, BAR_EPI = 26, BAR_ITEM = 28,
+       BAR_ITEMFREE = 30, BAR_COUNT = 32 };
+static_assert(8 * BAR_COUNT <= 256, "barrier block");
 
 template <int G>
 __global__ void __launch_bounds__(kPairThreads, 1)
@@ -75,10 +90,11 @@ rpa_tile2_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* smem = smem_raw + (smem_base - smem_u32(smem_raw));
     const uint32_t bars = smem_base + C::OFF_BAR;
-    volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem + C::OFF_BAR + 8 * BAR_COUNT);
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + C::OFF_BAR + 8 * BAR_COUNT + 8);
-    volatile int* progress = reinterpret_cast<volatile int*>(smem + C::OFF_BAR + 8 * BAR_COUNT + 16);
-    volatile int* item_slots = reinterpret_cast<volatile int*>(smem + C::OFF_BAR + 256);
+    volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem + C::OFF_FLAGS);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + C::OFF_FLAGS + 8);
+    // key blocks (counted across items) whose first PV product has been issued; written by the MMA warp
+    volatile int* progress = reinterpret_cast<volatile int*>(smem + C::OFF_FLAGS + 16);
+    volatile int* item_slots = reinterpret_cast<volatile int*>(smem + C::OFF_SLOTS);
     auto bar = [&](int slot) { return bars + 8u * slot; };
 
     if (a.validated && (*reinterpret_cast<volatile uint32_t*>(a.status) & kStatusBadInput)) return;  // inputs were rejected
@@ -89,15 +105,30 @@ rpa_tile2_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
     auto wait = [&](int slot, uint32_t parity, uint32_t code) {
         return mbar_wait_pair(bar(slot), parity, abort_flag, peer_abort, a.status, code);
     };
-    auto wait_for_item = [&](uint32_t code) {  // the next item's entry, written from the first CTA
-        return mbar_wait_pair<true>(bar(BAR_NEXT), 0, abort_flag, peer_abort, a.status, code);
-    };
     auto first_cta_bar = [&](int slot) { return map_to_cta(bar(slot), 0u); };
     const int ps = a.page_size;
+    const int n_items = a.num_tile_items;
     if (tid == 0) {
         *abort_flag = 0u;
-        mbar_init(bar(BAR_Q + 0), 1);
-        mbar_init(bar(BAR_Q + 1), 1);
+        *progress = 0;
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(bar(BAR_Q + s), 1);
+            mbar_init(bar(BAR_QPEER + s), 1);
+            mbar_init(bar(BAR_QFREE + s), 8);  // the softmax warps of this CTA, after an item's epilogue
+            mbar_init(bar(BAR_KFULL + s), 1);
+            mbar_init(bar(BAR_KEMPTY + s), 1);
+            mbar_init(bar(BAR_VFULL + s), 1);
+            mbar_init(bar(BAR_VEMPTY + s), 1);
+            mbar_init(bar(BAR_KPEER + s), 1);
+            mbar_init(bar(BAR_VPEER + s), 1);
+            mbar_init(bar(BAR_SFULL + s), 1);
+            mbar_init(bar(BAR_PREADY + s), 8);  // one arrival per softmax warp of the tile, both CTAs
+            mbar_init(bar(BAR_ODONE + s), 1);
+            mbar_init(bar(BAR_UPD + s), 1);
+            mbar_init(bar(BAR_EPI + s), 128);
+            mbar_init(bar(BAR_ITEM + s), 1);
+            mbar_init(bar(BAR_ITEMFREE + s), kPairWarps);  // every warp of both CTAs has read the slot
+        }
         fence_mbar_init();
     }
     if (warp == 1) {
@@ -111,222 +142,204 @@ rpa_tile2_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
     const uint32_t tm_s[2] = {tmem_base, tmem_base + 128u};
     const uint32_t tm_o[2] = {tmem_base + 256u, tmem_base + 256u + D};
 
-    // Pairs are persistent: the first CTA draws items from the device-wide counter (the list is
-    // sorted heaviest first) and writes each entry into both CTAs' item slots.
-    const int n_items = a.num_tile_items;
-    auto init_barriers = [&]() {
-        mbar_init(bar(BAR_NEXT), 1);
-        mbar_init(bar(BAR_QPEER), 1);
-        for (int s = 0; s < 2; ++s) {
-            mbar_init(bar(BAR_KFULL + s), 1);
-            mbar_init(bar(BAR_KEMPTY + s), 1);
-            mbar_init(bar(BAR_VFULL + s), 1);
-            mbar_init(bar(BAR_VEMPTY + s), 1);
-            mbar_init(bar(BAR_SFULL + s), 1);
-            mbar_init(bar(BAR_PREADY + s), 8);  // one arrival per softmax warp of the tile, both CTAs
-            mbar_init(bar(BAR_ODONE + s), 1);
-            mbar_init(bar(BAR_UPD + s), 1);
-            mbar_init(bar(BAR_EPI + s), 128);
-            mbar_init(bar(BAR_KPEER + s), 1);
-            mbar_init(bar(BAR_VPEER + s), 1);
-        }
-        fence_mbar_init();
-    };
-    // the entry of the item just fetched into `slot`, copied into the other CTA's slot (one thread)
-    auto send_item = [&](volatile int* slot) {
-        const uint32_t dst = map_to_cta(smem_u32(const_cast<int*>(slot)), 1u);
-        for (int k = 0; k < RAW_BOUNDS + 2; ++k) st_cluster_u32(dst + 4u * k, (uint32_t)slot[k]);
+    // Item n of this pair lives in slot n & 1.  A warp takes it (all lanes together): waits until the
+    // drawing warp has published it, reads it, and tells the drawing warp that this warp is done with
+    // the slot.  Returns false when the wait gave up.
+    auto take_item = [&](int n, TileCtx& it, int& item) -> bool {
+        const bool ok = mbar_wait_pair<true>(bar(BAR_ITEM + (n & 1)), (n >> 1) & 1, abort_flag, peer_abort, a.status, 0x60);
+        if (!__all_sync(0xffffffffu, ok)) return false;
+        const volatile int* slot = item_slots + (n & 1) * RAW_INTS;
+        item = slot[RAW_ITEM];
+        if (item < n_items) it = tile_ctx_from_raw(a, slot, kBlockN);
+        __syncwarp();
+        if (lane == 0) mbar_arrive_cluster(first_cta_bar(BAR_ITEMFREE + (n & 1)));
+        return true;
     };
     // this CTA's share of an item: its two query tiles' tokens
     auto own_tokens = [&](const TileCtx& it) { return max(0, min(2 * TQ, it.n_tok - (int)rank * 2 * TQ)); };
+    // valid positions of key block j of an item (the rest of the block is masked for every row)
+    auto valid_in_block = [&](const TileCtx& it, int j) {
+        return j < it.n_ctx_blocks ? min(kBlockN, it.c - j * kBlockN) : min(kBlockN, it.n_new_visible - (j - it.n_ctx_blocks) * kBlockN);
+    };
+    // rows of this CTA's V stage past the block's valid positions may hold stale or foreign
+    // data: make them finite (zero) so that masked probabilities (exactly 0) cannot produce NaN
+    auto zero_v_tail = [&](int n_valid, int st) {
+        if (n_valid < kBlockN) {
+            uint8_t* v_s = smem + C::OFF_V + st * C::V_STAGE;
+            for (int idx = lane; idx < (kBlockN - n_valid) * 8; idx += 32)
+                *reinterpret_cast<uint4*>(v_s + (n_valid + idx / 8) * 128 + (idx % 8) * 16) = make_uint4(0, 0, 0, 0);
+            fence_proxy_async_smem();
+            __syncwarp();
+        }
+    };
 
     if (warp < 4) {
-      // first warpgroup: producer, MMA issuer / relay, cache update; it needs few registers
+      // first warpgroup: producer, MMA issuer / relay, cache update and item drawing; it needs few registers
       asm volatile("setmaxnreg.dec.sync.aligned.u32 56;\n");
-      int q_prefetched_for = -1;  // producer: the iteration whose query tiles are already on their way
-      for (int iter = 0;; ++iter) {
-      tc_fence_before();
-      cluster_sync();  // both CTAs are done with the previous item
-      if (*abort_flag) break;
-      volatile int* slot = item_slots + (iter & 1) * RAW_INTS;
-      if (iter == 0 && first_cta && warp == 0) {
-          draw_and_fetch_tile(a, true, 0, slot, lane);
-          __syncwarp();
-          if (lane == 0) send_item(slot);
-      }
-      if (tid == 0) {
-          init_barriers();
-          *progress = 0;
-      }
-      cluster_sync();  // item slots filled and both CTAs' mbarriers re-initialised
-      tc_fence_after();
-      if (slot[RAW_ITEM] >= n_items) break;
-      const TileCtx it = tile_ctx_from_raw(a, slot, kBlockN);
-      if (!debug_rows_ok(a, (long long)it.cu + it.q_tok0, it.n_tok)) break;  // (bounds-checked build: both CTAs take this exit together)
-      const int h = it.h, cu = it.cu, c = it.c;
-      const int n_ctx_blocks = it.n_ctx_blocks, n_new_visible = it.n_new_visible, n_blocks = it.n_blocks;
-      const int32_t* pt_row = it.pt_row;
-      const uint32_t q_region = smem_base + C::OFF_Q + (iter & 1) * 2 * C::TILE_BYTES;
-      // valid positions of key block j (the rest of the block is masked for every row)
-      auto valid_in_block = [&](int j) {
-          return j < n_ctx_blocks ? min(kBlockN, c - j * kBlockN) : min(kBlockN, n_new_visible - (j - n_ctx_blocks) * kBlockN);
-      };
-      // rows of this CTA's V stage past the block's valid positions may hold stale or foreign
-      // data: make them finite (zero) so that masked probabilities (exactly 0) cannot produce NaN
-      auto zero_v_tail = [&](int j) {
-          const int n_valid = valid_in_block(j);
-          if (n_valid < kBlockN) {
-              uint8_t* v_s = smem + C::OFF_V + (j & 1) * C::V_STAGE;
-              for (int idx = lane; idx < (kBlockN - n_valid) * 8; idx += 32)
-                  *reinterpret_cast<uint4*>(v_s + (n_valid + idx / 8) * 128 + (idx % 8) * 16) = make_uint4(0, 0, 0, 0);
-              fence_proxy_async_smem();
-              __syncwarp();
-          }
-      };
       if (warp == 0) {
         // ================================ TMA producer (each CTA: its own halves) ================================
-        auto load_q = [&](uint32_t region, uint32_t q_bar, int head, int tok_row) {  // one thread
-            if (a.ablation & kAblateLoads) {
-                mbar_arrive(q_bar);
-                return;
-            }
-            mbar_arrive_expect_tx(q_bar, 2 * C::TILE_BYTES);  // (rows past the tensors read as zero and count)
-            for (int x = 0; x < 2; ++x)
-#pragma unroll
-                for (int b = 0; b < C::NBLK; ++b)
-                    tma_load_3d(region + x * C::TILE_BYTES + b * C::BLK_BYTES, &maps.q, b * 64, head * G, tok_row + x * TQ, q_bar);
-        };
         if (lane == 0) {
             prefetch_tmap(&maps.q);
             prefetch_tmap(&maps.out);
             prefetch_tmap(&maps.cache);
             prefetch_tmap(&maps.new_k);
             prefetch_tmap(&maps.new_v);
-            if (q_prefetched_for != iter) load_q(q_region, bar(BAR_Q + (iter & 1)), h, cu + it.q_tok0 + (int)rank * 2 * TQ);
         }
         const int box_rows = page_box_rows(ps, kHalfN);
+        int gb = 0;  // key blocks of earlier items: block j of the running item is fill gb + j of either ring
         bool ok = true;
-        // fills stage j & 1 of the K (kv = 0) or V (kv = 1) ring with this CTA's half of block j:
-        // keys [64 rank, 64 rank + 64) of the block with all of d_k, or all 128 positions of V with
-        // columns [64 rank, 64 rank + 64)
-        auto fill = [&](int j, int kv) -> bool {
-            const bool ctx = j < n_ctx_blocks;
-            const int st = j & 1;
-            if (!debug_stage_ok(a, st, C::KS)) return false;
-            const int rows = kv ? kBlockN : kHalfN;            // rows of the block this CTA stages
-            const int row0 = kv ? 0 : (int)rank * kHalfN;      // ... starting at this row of the block
-            const int boxes = rows / box_rows;
-            int page = 0, slot0 = 0;
-            bool sub_valid = false;
-            if (ctx) {
-                const int pos = j * kBlockN + row0 + lane * box_rows;
-                sub_valid = lane < boxes && pos < c;
-                if (sub_valid) {
-                    page = debug_read_page(a, pt_row[pos / ps]);
-                    slot0 = pos % ps;
+        for (int n = 0; ok; ++n) {
+            TileCtx it;
+            int item;
+            ok = take_item(n, it, item);
+            if (!ok || item >= n_items) break;
+            if (!debug_rows_ok(a, (long long)it.cu + it.q_tok0, it.n_tok)) break;
+            const int h = it.h, cu = it.cu, c = it.c, n_ctx_blocks = it.n_ctx_blocks, n_blocks = it.n_blocks;
+            const int32_t* pt_row = it.pt_row;
+            // the item's query tiles, into the buffer the item before the last one has left
+            if (n >= 2) ok = wait(BAR_QFREE + (n & 1), ((n >> 1) - 1) & 1, 0x15);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            if (lane == 0) {
+                const uint32_t region = smem_base + C::OFF_Q + (n & 1) * 2 * C::TILE_BYTES, q_bar = bar(BAR_Q + (n & 1));
+                const int tok_row = cu + it.q_tok0 + (int)rank * 2 * TQ;
+                if (a.ablation & kAblateLoads) {
+                    mbar_arrive(q_bar);
+                } else {
+                    mbar_arrive_expect_tx(q_bar, 2 * C::TILE_BYTES);  // (rows past the tensors read as zero and count)
+                    for (int x = 0; x < 2; ++x)
+#pragma unroll
+                        for (int b = 0; b < C::NBLK; ++b)
+                            tma_load_3d(region + x * C::TILE_BYTES + b * C::BLK_BYTES, &maps.q, b * 64, h * G, tok_row + x * TQ, q_bar);
                 }
             }
-            const int n_sub_valid = __popc(__ballot_sync(0xffffffffu, sub_valid));
-            const uint32_t bytes = ctx ? (uint32_t)n_sub_valid * box_rows * 128u * (kv ? 1u : (uint32_t)C::NBLK)
-                                       : (uint32_t)(kv ? C::V_STAGE : C::K_STAGE);
-            const int full = (kv ? BAR_VFULL : BAR_KFULL) + st, empty = (kv ? BAR_VEMPTY : BAR_KEMPTY) + st;
-            bool good = true;
-            if (j >= 2) good = wait(empty, ((j >> 1) - 1) & 1, 0x10 + kv);
-            good = __all_sync(0xffffffffu, good);
-            if (!good) return false;
-            const uint32_t dst = smem_base + (kv ? C::OFF_V + st * C::V_STAGE : C::OFF_K + st * C::K_STAGE);
-            if (a.ablation & kAblateLoads) {
-                if (lane == 0) mbar_arrive(bar(full));
-                return true;
-            }
-            if (lane == 0) mbar_arrive_expect_tx(bar(full), bytes);  // (0 bytes: completes at once)
-            __syncwarp();
-            if (ctx) {
-                if (sub_valid) {
+            // fills the next stage of the K (kv = 0) or V (kv = 1) ring with this CTA's half of block j:
+            // keys [64 rank, 64 rank + 64) of the block with all of d_k, or all 128 positions of V with
+            // columns [64 rank, 64 rank + 64)
+            auto fill = [&](int j, int kv) -> bool {
+                const bool ctx = j < n_ctx_blocks;
+                const int f = gb + j, st = f & 1;
+                if (!debug_stage_ok(a, st, C::KS)) return false;
+                const int rows = kv ? kBlockN : kHalfN;            // rows of the block this CTA stages
+                const int row0 = kv ? 0 : (int)rank * kHalfN;      // ... starting at this row of the block
+                const int boxes = rows / box_rows;
+                int page = 0, slot0 = 0;
+                bool sub_valid = false;
+                if (ctx) {
+                    const int pos = j * kBlockN + row0 + lane * box_rows;
+                    sub_valid = lane < boxes && pos < c;
+                    if (sub_valid) {
+                        page = debug_read_page(a, pt_row[pos / ps]);
+                        slot0 = pos % ps;
+                    }
+                }
+                const int n_sub_valid = __popc(__ballot_sync(0xffffffffu, sub_valid));
+                const uint32_t bytes = ctx ? (uint32_t)n_sub_valid * box_rows * 128u * (kv ? 1u : (uint32_t)C::NBLK)
+                                           : (uint32_t)(kv ? C::V_STAGE : C::K_STAGE);
+                const int full = (kv ? BAR_VFULL : BAR_KFULL) + st, empty = (kv ? BAR_VEMPTY : BAR_KEMPTY) + st;
+                bool good = true;
+                if (f >= 2) good = wait(empty, ((f >> 1) - 1) & 1, 0x10 + kv);
+                good = __all_sync(0xffffffffu, good);
+                if (!good) return false;
+                const uint32_t dst = smem_base + (kv ? C::OFF_V + st * C::V_STAGE : C::OFF_K + st * C::K_STAGE);
+                if (a.ablation & kAblateLoads) {
+                    if (lane == 0) mbar_arrive(bar(full));
+                    return true;
+                }
+                if (lane == 0) mbar_arrive_expect_tx(bar(full), bytes);  // (0 bytes: completes at once)
+                __syncwarp();
+                if (ctx) {
+                    if (sub_valid) {
+                        if (kv) {
+                            tma_load_4d(dst + lane * box_rows * 128, &maps.cache, (int)rank * 64, 2 * h + 1, slot0, page, bar(full));
+                        } else {
+#pragma unroll
+                            for (int b = 0; b < C::NBLK; ++b)
+                                tma_load_4d(dst + b * C::HALF_BLK + lane * box_rows * 128, &maps.cache, b * 64, 2 * h, slot0, page, bar(full));
+                        }
+                    }
+                } else if (lane == 0) {
+                    const int new_row0 = cu + (j - n_ctx_blocks) * kBlockN;
                     if (kv) {
-                        tma_load_4d(dst + lane * box_rows * 128, &maps.cache, (int)rank * 64, 2 * h + 1, slot0, page, bar(full));
+#pragma unroll
+                        for (int i = 0; i < kBlockN / kHalfN; ++i)
+                            tma_load_3d(dst + i * C::HALF_BLK, &maps.new_v, (int)rank * 64, h, new_row0 + i * kHalfN, bar(full));
                     } else {
 #pragma unroll
                         for (int b = 0; b < C::NBLK; ++b)
-                            tma_load_4d(dst + b * C::HALF_BLK + lane * box_rows * 128, &maps.cache, b * 64, 2 * h, slot0, page, bar(full));
+                            tma_load_3d(dst + b * C::HALF_BLK, &maps.new_k, b * 64, h, new_row0 + (int)rank * kHalfN, bar(full));
                     }
                 }
-            } else if (lane == 0) {
-                const int new_row0 = cu + (j - n_ctx_blocks) * kBlockN;
-                if (kv) {
-#pragma unroll
-                    for (int i = 0; i < kBlockN / kHalfN; ++i)
-                        tma_load_3d(dst + i * C::HALF_BLK, &maps.new_v, (int)rank * 64, h, new_row0 + i * kHalfN, bar(full));
-                } else {
-#pragma unroll
-                    for (int b = 0; b < C::NBLK; ++b)
-                        tma_load_3d(dst + b * C::HALF_BLK, &maps.new_k, b * 64, h, new_row0 + (int)rank * kHalfN, bar(full));
-                }
+                return true;
+            };
+            // the keys run one block ahead of the values (a V stage is held through its block's whole softmax)
+            for (int t = 0; t <= n_blocks && ok; ++t) {
+                if (t < n_blocks) ok = fill(t, 0);
+                if (ok && t >= 1) ok = fill(t - 1, 1);
             }
-            return true;
-        };
-        // the keys run one block ahead of the values (a V stage is held through its block's whole softmax)
-        for (int t = 0; t <= n_blocks && ok; ++t) {
-            if (t < n_blocks) ok = fill(t, 0);
-            if (ok && t >= 1) ok = fill(t - 1, 1);
+            gb += n_blocks;
         }
-        // the next item's query tiles go into the other buffer (free since the cluster barrier above)
-        if (ok) ok = wait_for_item(0x12);
-        const volatile int* nxt = item_slots + ((iter + 1) & 1) * RAW_INTS;
-        if (ok && nxt[RAW_ITEM] < n_items) {
-            if (lane == 0)
-                load_q(smem_base + C::OFF_Q + ((iter + 1) & 1) * 2 * C::TILE_BYTES, bar(BAR_Q + ((iter + 1) & 1)), nxt[RAW_HEAD],
-                       nxt[RAW_CU] + nxt[RAW_TOK0] + (int)rank * 2 * TQ);
-            q_prefetched_for = iter + 1;
-        }
-        // every completion signal of this item's products has reached this CTA before it goes round
+        // every completion signal of the products has reached this CTA before it leaves
 #pragma unroll
         for (int st = 0; st < 2; ++st) {
-            const int uses = (n_blocks + 1 - st) >> 1;  // key blocks of this item that went through stage st
+            const int uses = (gb + 1 - st) >> 1;  // fills that went through stage st
             if (uses > 0 && ok) ok = wait(BAR_KEMPTY + st, (uses - 1) & 1, 0x13);
             if (uses > 0 && ok) ok = wait(BAR_VEMPTY + st, (uses - 1) & 1, 0x14);
         }
       } else if (warp == 1 && !first_cta) {
         // ================================ second CTA: relay "my half has landed" ================================
-        bool ok = wait(BAR_Q + (iter & 1), (iter >> 1) & 1, 0x28);
-        if (ok && lane == 0) mbar_arrive_cluster(first_cta_bar(BAR_QPEER));
-        for (int t = 0; t <= n_blocks && ok; ++t) {
-            if (t < n_blocks) {
-                ok = wait(BAR_KFULL + (t & 1), (t >> 1) & 1, 0x29);
-                if (ok && lane == 0) mbar_arrive_cluster(first_cta_bar(BAR_KPEER + (t & 1)));
-            }
-            if (ok && t >= 1) {
-                const int j = t - 1;
-                ok = wait(BAR_VFULL + (j & 1), (j >> 1) & 1, 0x2A);
-                if (ok) {
-                    zero_v_tail(j);
-                    if (lane == 0) {
-                        if (valid_in_block(j) < kBlockN) {
-                            mbar_arrive_cluster_release(first_cta_bar(BAR_VPEER + (j & 1)));  // the zeroed rows count
-                        } else {
-                            mbar_arrive_cluster(first_cta_bar(BAR_VPEER + (j & 1)));
+        int gb = 0;
+        bool ok = true;
+        for (int n = 0; ok; ++n) {
+            TileCtx it;
+            int item;
+            ok = take_item(n, it, item);
+            if (!ok || item >= n_items) break;
+            if (!debug_rows_ok(a, (long long)it.cu + it.q_tok0, it.n_tok)) break;
+            const int n_blocks = it.n_blocks;
+            ok = wait(BAR_Q + (n & 1), (n >> 1) & 1, 0x28);
+            if (ok && lane == 0) mbar_arrive_cluster(first_cta_bar(BAR_QPEER + (n & 1)));
+            for (int t = 0; t <= n_blocks && ok; ++t) {
+                if (t < n_blocks) {
+                    const int f = gb + t;
+                    ok = wait(BAR_KFULL + (f & 1), (f >> 1) & 1, 0x29);
+                    if (ok && lane == 0) mbar_arrive_cluster(first_cta_bar(BAR_KPEER + (f & 1)));
+                }
+                if (ok && t >= 1) {
+                    const int f = gb + t - 1, n_valid = valid_in_block(it, t - 1);
+                    ok = wait(BAR_VFULL + (f & 1), (f >> 1) & 1, 0x2A);
+                    if (ok) {
+                        zero_v_tail(n_valid, f & 1);
+                        if (lane == 0) {
+                            if (n_valid < kBlockN) {
+                                mbar_arrive_cluster_release(first_cta_bar(BAR_VPEER + (f & 1)));  // the zeroed rows count
+                            } else {
+                                mbar_arrive_cluster(first_cta_bar(BAR_VPEER + (f & 1)));
+                            }
                         }
                     }
                 }
             }
+            gb += n_blocks;
         }
       } else if (warp == 1) {
         // ================================ MMA issuer (first CTA, for the pair) ================================
         constexpr uint32_t idesc_qk = instr_desc_bf16(256, kBlockN, 0, 0);
         constexpr uint32_t idesc_pv = instr_desc_bf16(256, D, 0, 1);
         constexpr uint32_t desc_hi = smem_desc_sw128_hi(1024);
-        const uint32_t q_lo[2] = {smem_desc_sw128_lo(q_region, 16), smem_desc_sw128_lo(q_region + C::TILE_BYTES, 16)};
         const uint32_t k_lo = smem_desc_sw128_lo(smem_base + C::OFF_K, 16);
         const uint32_t v_lo = smem_desc_sw128_lo(smem_base + C::OFF_V, C::BLK_BYTES);
         const bool no_compute = a.ablation & kAblateCompute;  // bench switch: commits without products
-        auto issue_qk = [&](int x, int st) {  // S_x = Q_x K^T over d_k in steps of 16, both CTAs' tile x
+        // S_x = Q_x K^T over d_k in steps of 16, tile x of both CTAs; the queries of item n, the keys in stage st
+        auto issue_qk = [&](int n, int x, int st) {
             if (no_compute) return;
+            const uint32_t ql = smem_desc_sw128_lo(smem_base + C::OFF_Q + ((n & 1) * 2 + x) * C::TILE_BYTES, 16);
             const uint32_t kl = k_lo + st * (C::K_STAGE >> 4);
 #pragma unroll
             for (int ks = 0; ks < D / 16; ++ks) {
                 const uint32_t q_off = ((ks / 4) * C::BLK_BYTES + (ks % 4) * 32) >> 4;
                 const uint32_t k_off = ((ks / 4) * C::HALF_BLK + (ks % 4) * 32) >> 4;
-                umma_ss_pair(tm_s[x], make_desc(q_lo[x] + q_off, desc_hi), make_desc(kl + k_off, desc_hi), idesc_qk, ks > 0);
+                umma_ss_pair(tm_s[x], make_desc(ql + q_off, desc_hi), make_desc(kl + k_off, desc_hi), idesc_qk, ks > 0);
             }
         };
         auto issue_pv = [&](int x, int st, bool first) {  // O_x (+)= P_x V over 128 positions in steps of 16
@@ -336,127 +349,169 @@ rpa_tile2_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
             for (int kk = 0; kk < kBlockN / 16; ++kk)
                 umma_ts_pair(tm_o[x], tm_s[x] + kk * 8, make_desc(vl + kk * (2048 >> 4), desc_hi), idesc_pv, !(first && kk == 0));
         };
-        auto k_landed = [&](int j, uint32_t code) {
-            return wait(BAR_KFULL + (j & 1), (j >> 1) & 1, code) && wait(BAR_KPEER + (j & 1), (j >> 1) & 1, code + 1);
+        auto q_landed = [&](int n) {
+            return wait(BAR_Q + (n & 1), (n >> 1) & 1, 0x20) && wait(BAR_QPEER + (n & 1), (n >> 1) & 1, 0x21);
         };
-        bool ok = wait(BAR_Q + (iter & 1), (iter >> 1) & 1, 0x20) && wait(BAR_QPEER, 0, 0x21);
-        ok = ok && k_landed(0, 0x22);
-        if (ok) {
-            tc_fence_after();
-            if (elect_one()) {
-                issue_qk(0, 0);
-                tc_commit_pair(bar(BAR_SFULL + 0));
-                issue_qk(1, 0);
-                tc_commit_pair(bar(BAR_SFULL + 1));
-                tc_commit_pair(bar(BAR_KEMPTY + 0));
-            }
-            __syncwarp();
-        }
-        for (int j = 0; j < n_blocks && ok; ++j) {
-            const int st = j & 1, ph = (j >> 1) & 1;
-            ok = wait(BAR_VFULL + st, ph, 0x24);
-            if (!ok) break;
-            zero_v_tail(j);
-            ok = wait(BAR_VPEER + st, ph, 0x25);
-            if (!ok) break;
-            const bool more = j + 1 < n_blocks;
-            const int st1 = (j + 1) & 1;
-            ok = wait(BAR_PREADY + 0, j & 1, 0x26);
-            if (!ok) break;
-            tc_fence_after();
-            if (elect_one()) {
-                issue_pv(0, st, j == 0);
-                tc_commit_pair(bar(BAR_ODONE + 0));
-                *progress = j + 1;
-            }
-            __syncwarp();
-            if (more) {
-                ok = k_landed(j + 1, 0x2C);
-                if (!ok) break;
+        auto k_landed = [&](int f, uint32_t code) {  // fill f of the K ring, both halves
+            return wait(BAR_KFULL + (f & 1), (f >> 1) & 1, code) && wait(BAR_KPEER + (f & 1), (f >> 1) & 1, code + 1);
+        };
+        int gb = 0;
+        TileCtx it, nxt;
+        int item, nxt_item = n_items;
+        bool ok = take_item(0, it, item);
+        if (ok && item < n_items && debug_rows_ok(a, (long long)it.cu + it.q_tok0, it.n_tok)) {
+            // the first item's first block; every later one is issued behind its predecessor's products
+            ok = q_landed(0) && k_landed(0, 0x22);
+            if (ok) {
                 tc_fence_after();
                 if (elect_one()) {
-                    issue_qk(0, st1);
+                    issue_qk(0, 0, 0);
                     tc_commit_pair(bar(BAR_SFULL + 0));
+                    issue_qk(0, 1, 0);
+                    tc_commit_pair(bar(BAR_SFULL + 1));
+                    tc_commit_pair(bar(BAR_KEMPTY + 0));
                 }
                 __syncwarp();
             }
-            ok = wait(BAR_PREADY + 1, j & 1, 0x27);
-            if (!ok) break;
-            tc_fence_after();
-            if (elect_one()) {
-                issue_pv(1, st, j == 0);
-                tc_commit_pair(bar(BAR_ODONE + 1));
-                tc_commit_pair(bar(BAR_VEMPTY + st));
-                if (more) {
-                    issue_qk(1, st1);
-                    tc_commit_pair(bar(BAR_SFULL + 1));
-                    tc_commit_pair(bar(BAR_KEMPTY + st1));
+            for (int n = 0; ok; ++n) {
+                const int n_blocks = it.n_blocks;
+                bool have_next = false, looked = false;
+                for (int j = 0; j < n_blocks && ok; ++j) {
+                    const int f = gb + j, st = f & 1, ph = (f >> 1) & 1;
+                    ok = wait(BAR_VFULL + st, ph, 0x24);
+                    if (!ok) break;
+                    zero_v_tail(valid_in_block(it, j), st);
+                    ok = wait(BAR_VPEER + st, ph, 0x25);
+                    if (!ok) break;
+                    const bool last = j + 1 == n_blocks;
+                    ok = wait(BAR_PREADY + 0, f & 1, 0x26);
+                    if (!ok) break;
+                    tc_fence_after();
+                    if (elect_one()) {
+                        issue_pv(0, st, j == 0);
+                        tc_commit_pair(bar(BAR_ODONE + 0));
+                        *progress = f + 1;
+                    }
+                    __syncwarp();
+                    if (last && !looked) {  // what follows this item?  (drawn by now: the drawing warp watches `progress`)
+                        looked = true;
+                        ok = take_item(n + 1, nxt, nxt_item);
+                        if (!ok) break;
+                        have_next = nxt_item < n_items && debug_rows_ok(a, (long long)nxt.cu + nxt.q_tok0, nxt.n_tok);
+                    }
+                    // the next score product of tile A: the item's next block, or the next item's first one
+                    const bool more = !last || have_next;
+                    const int f1 = f + 1, st1 = f1 & 1, n1 = last ? n + 1 : n;
+                    if (more) {
+                        if (last) ok = q_landed(n + 1);
+                        ok = ok && k_landed(f1, 0x2C);
+                        if (!ok) break;
+                        tc_fence_after();
+                        if (elect_one()) {
+                            issue_qk(n1, 0, st1);
+                            tc_commit_pair(bar(BAR_SFULL + 0));
+                        }
+                        __syncwarp();
+                    }
+                    ok = wait(BAR_PREADY + 1, f & 1, 0x27);
+                    if (!ok) break;
+                    tc_fence_after();
+                    if (elect_one()) {
+                        issue_pv(1, st, j == 0);
+                        tc_commit_pair(bar(BAR_ODONE + 1));
+                        tc_commit_pair(bar(BAR_VEMPTY + st));
+                        if (more) {
+                            issue_qk(n1, 1, st1);
+                            tc_commit_pair(bar(BAR_SFULL + 1));
+                            tc_commit_pair(bar(BAR_KEMPTY + st1));
+                        }
+                    }
+                    __syncwarp();
                 }
+                gb += n_blocks;
+                if (!have_next) break;
+                it = nxt;
             }
-            __syncwarp();
         }
       } else {
-        // ================================ fused cache update (each CTA: its own tokens) ================================
-        // In the first CTA one warp also draws the pair's next item - once the running one is within
-        // two key blocks of its end, so that no long item is reserved early - and hands it to both CTAs.
-        auto fetch_next = [&]() {
+        // ================================ fused cache update (each CTA: its own tokens); item drawing ================================
+        // Warp 3 of the first CTA draws the pair's items - the next one once the running one is within
+        // a few key blocks of its end, so that no long item is reserved early - and writes each entry
+        // into both CTAs' slots.
+        auto publish = [&](int n, int fallback) {  // whole warp
+            bool ok = true;
+            if (n >= 2) ok = wait(BAR_ITEMFREE + (n & 1), ((n >> 1) - 1) & 1, 0x61);
+            if (!__all_sync(0xffffffffu, ok)) return false;
+            volatile int* slot = item_slots + (n & 1) * RAW_INTS;
+            draw_and_fetch_tile(a, true, fallback, slot, lane);
+            __syncwarp();
             if (lane == 0) {
-                const long long t0 = clock64();
-                while (*progress < n_blocks - 2 && !*abort_flag && clock64() - t0 < 2000000000LL) __nanosleep(256);
+                const uint32_t dst = map_to_cta(smem_u32(const_cast<int*>(slot)), 1u);
+                for (int k = 0; k < RAW_BOUNDS + 2; ++k) st_cluster_u32(dst + 4u * k, (uint32_t)slot[k]);
+                mbar_arrive(bar(BAR_ITEM + (n & 1)));
+                mbar_arrive_cluster_release(map_to_cta(bar(BAR_ITEM + (n & 1)), 1u));  // the entry written above is visible to its waiters
             }
             __syncwarp();
-            volatile int* nxt = item_slots + ((iter + 1) & 1) * RAW_INTS;
-            draw_and_fetch_tile(a, true, n_items, nxt, lane);
-            __syncwarp();
-            if (lane == 0) {
-                send_item(nxt);
-                mbar_arrive(bar(BAR_NEXT));
-                mbar_arrive_cluster_release(map_to_cta(bar(BAR_NEXT), 1u));  // the entry written above is visible to its waiter
-            }
+            return true;
         };
-        const bool fetch_early = n_blocks <= 2;
-        if (warp == 3 && first_cta && fetch_early) fetch_next();
-        if (!(a.ablation & kAblateUpdate) && (it.flags & kFlagWriteKv)) {
-            TileCtx own = it;
-            own.q_tok0 = it.q_tok0 + (int)rank * 2 * TQ;
-            own.n_tok = own_tokens(it);
-            tile_update_cache<D>(a, own, warp - 2, lane, smem_base + C::OFF_UPD, bar(BAR_UPD + warp - 2), abort_flag, a.status);
+        const bool drawer = warp == 3 && first_cta;
+        int gb = 0, upd_rounds = 0;
+        bool ok = true;
+        if (drawer) ok = publish(0, 0);
+        for (int n = 0; ok; ++n) {
+            TileCtx it;
+            int item;
+            ok = take_item(n, it, item);
+            if (!ok || item >= n_items) break;
+            if (!debug_rows_ok(a, (long long)it.cu + it.q_tok0, it.n_tok)) break;
+            if (!(a.ablation & kAblateUpdate) && (it.flags & kFlagWriteKv)) {
+                TileCtx own = it;
+                own.q_tok0 = it.q_tok0 + (int)rank * 2 * TQ;
+                own.n_tok = own_tokens(it);
+                ok = tile_update_cache<D>(a, own, warp - 2, lane, smem_base + C::OFF_UPD, bar(BAR_UPD + warp - 2), abort_flag, a.status,
+                                          &upd_rounds);
+            }
+            if (drawer && ok) {
+                if (lane == 0) {
+                    const long long t0 = clock64();
+                    while (*progress < gb + it.n_blocks - kFetchAhead && !*abort_flag && clock64() - t0 < 4000000000LL) __nanosleep(256);
+                }
+                __syncwarp();
+                ok = publish(n + 1, n_items);
+            }
+            gb += it.n_blocks;
         }
-        if (warp == 3 && first_cta && !fetch_early) fetch_next();
       }
-      }  // item loop of the first warpgroup
     } else {
         // ================================ softmax warps ================================
         asm volatile("setmaxnreg.inc.sync.aligned.u32 224;\n");
-        for (int iter = 0;; ++iter) {
-        tc_fence_before();
-        cluster_sync();  // both CTAs are done with the previous item
-        if (*abort_flag) break;
-        cluster_sync();  // item slots filled and mbarriers re-initialised
-        tc_fence_after();
-        const volatile int* slot = item_slots + (iter & 1) * RAW_INTS;
-        if (slot[RAW_ITEM] >= n_items) break;
-        const TileCtx it = tile_ctx_from_raw(a, slot, kBlockN);
-        if (!debug_rows_ok(a, (long long)it.cu + it.q_tok0, it.n_tok)) break;
-        const int h = it.h, cu = it.cu, q_r = it.q_r, L = it.L, c = it.c;
-        const int n_ctx_blocks = it.n_ctx_blocks, n_new_visible = it.n_new_visible, n_blocks = it.n_blocks;
-        const uint32_t q_region = smem_base + C::OFF_Q + (iter & 1) * 2 * C::TILE_BYTES;
         const int x = (warp - 4) >> 2;              // 0: tile A, 1: tile B
         const int quarter = warp & 3;               // TMEM lanes this warp may touch: 32*quarter ..
         const int row = quarter * 32 + lane;        // query row of this thread inside its tile
         const int tok_in_tile = row / G, g = row % G;
         const int tok_in_item = ((int)rank * 2 + x) * TQ + tok_in_tile;
-        const int tok = it.q_tok0 + tok_in_item;    // token index inside the sequence
-        const bool row_valid = tok_in_item < it.n_tok;
         const uint32_t lane_sel = (uint32_t)(quarter * 32) << 16;
         const uint32_t s_addr = tm_s[x] + lane_sel, o_addr = tm_o[x] + lane_sel;
-        const int lim = a.causal ? c + min(tok, q_r - 1) : L - 1;  // last visible key position of this row
         const uint32_t pready = first_cta ? bar(BAR_PREADY + x) : first_cta_bar(BAR_PREADY + x);
+        int gb = 0, epi_uses = 0;
+        bool ok = true;
+        for (int n = 0; ok; ++n) {
+        TileCtx it;
+        int item;
+        ok = take_item(n, it, item);
+        if (!ok || item >= n_items) break;
+        if (!debug_rows_ok(a, (long long)it.cu + it.q_tok0, it.n_tok)) break;
+        const int h = it.h, cu = it.cu, q_r = it.q_r, L = it.L, c = it.c;
+        const int n_ctx_blocks = it.n_ctx_blocks, n_new_visible = it.n_new_visible, n_blocks = it.n_blocks;
+        const uint32_t q_region = smem_base + C::OFF_Q + (n & 1) * 2 * C::TILE_BYTES;
+        const int tok = it.q_tok0 + tok_in_item;    // token index inside the sequence
+        const bool row_valid = tok_in_item < it.n_tok;
+        const int lim = a.causal ? c + min(tok, q_r - 1) : L - 1;  // last visible key position of this row
 
         float m_ref = -INFINITY, l_sum = 0.f;
-        bool ok = true;
         for (int j = 0; j < n_blocks; ++j) {
-            ok = wait(BAR_SFULL + x, j & 1, 0x30 + x);
+            const int f = gb + j;
+            ok = wait(BAR_SFULL + x, f & 1, 0x30 + x);
             if (!ok) break;
             tc_fence_after();
             if (a.ablation & kAblateCompute) {  // bench switch: hand over at once
@@ -499,20 +554,20 @@ rpa_tile2_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
                 const bool grow = mx2 - m_ref > kRescaleThreshold;
                 if (__any_sync(0xffffffffu, grow)) {
                     // the previous PV product of this tile must have landed before O is touched
-                    ok = wait(BAR_ODONE + x, (j - 1) & 1, 0x32 + x);
+                    ok = wait(BAR_ODONE + x, (f - 1) & 1, 0x32 + x);
                     if (!ok) break;
                     tc_fence_after();
-                    const float f = grow ? fast_exp2(m_ref - mx2) : 1.f;
+                    const float fs = grow ? fast_exp2(m_ref - mx2) : 1.f;
 #pragma unroll
                     for (int ch = 0; ch < D / 32; ++ch) {
                         uint32_t r32[32];
                         tmem_ld32(o_addr + ch * 32, r32);
                         tc_wait_ld();
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) r32[i] = __float_as_uint(__uint_as_float(r32[i]) * f);
+                        for (int i = 0; i < 32; ++i) r32[i] = __float_as_uint(__uint_as_float(r32[i]) * fs);
                         tmem_st32(o_addr + ch * 32, r32);
                     }
-                    l_sum *= f;
+                    l_sum *= fs;
                     if (grow) m_ref = mx2;
                 }
             }
@@ -539,14 +594,13 @@ rpa_tile2_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
             if (lane == 0) mbar_arrive_cluster(pready);  // one arrival per warp, at the first CTA's barrier
         }
         // ---- epilogue: O / l -> bf16 -> out ----
-        if (ok && n_blocks > 0) ok = wait(BAR_ODONE + x, (n_blocks - 1) & 1, 0x34 + x);
-        if (a.ablation & kAblateCompute) ok = false;  // nothing to write
-        if (ok && n_blocks > 0) {
+        if (ok && n_blocks > 0) ok = wait(BAR_ODONE + x, (gb + n_blocks - 1) & 1, 0x34 + x);
+        if (ok && n_blocks > 0 && !(a.ablation & kAblateCompute)) {
             tc_fence_after();
             const float inv = a.out_scale / l_sum;
             if (((int)rank * 2 + x + 1) * TQ <= it.n_tok) {
                 // A full tile goes out through shared memory: each thread parks its row in the
-                // tile's Q buffer (free since the last score product completed) in the swizzled
+                // tile's Q buffer (free since the item's last score product completed) in the swizzled
                 // layout of the tensor map, and one thread stores the tile with the copy engine.
                 const uint32_t q_buf = q_region + x * C::TILE_BYTES;
 #pragma unroll
@@ -567,7 +621,7 @@ rpa_tile2_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
                 fence_proxy_async_smem();
                 mbar_arrive(bar(BAR_EPI + x));
                 if (row == 0) {
-                    if (wait(BAR_EPI + x, 0, 0x36 + x)) {
+                    if (wait(BAR_EPI + x, epi_uses & 1, 0x36 + x)) {
 #pragma unroll
                         for (int b = 0; b < C::NBLK; ++b)
                             tma_store_3d(&maps.out, q_buf + b * C::BLK_BYTES, b * 64, h * G, cu + it.q_tok0 + ((int)rank * 2 + x) * TQ);
@@ -575,6 +629,7 @@ rpa_tile2_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
                         bulk_wait_read();  // the Q buffer is loaded again two items later
                     }
                 }
+                ++epi_uses;
             } else {
                 uint16_t* dst = a.out + (((int64_t)cu + tok) * a.h_q + h * G + g) * D;
 #pragma unroll
@@ -596,6 +651,13 @@ rpa_tile2_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
                 }
             }
         }
+        // this warp is done with the item's query buffer (the producer loads the item after next into it)
+        // and with the accumulator (the next item's first PV product overwrites it once this warp has
+        // handed over that item's first probabilities)
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar(BAR_QFREE + (n & 1)));
+        gb += n_blocks;
         }  // item loop of the softmax warpgroups
     }
     // ---- teardown: both CTAs arrive, then each frees its half of the pair's TMEM allocation ----

@@ -120,7 +120,8 @@ __device__ __forceinline__ int packed_seq_of(const TileCtx& it, int tok) {
 // token's K row and V row into the warp's staging area (completion on the warp's mbarrier `bar`),
 // then writes both with one bulk store, since K_h and V_h are neighbours in a cache slot.  Plain
 // loads and stores would queue behind the epilogue's stores in the load/store unit and hold a short
-// item back by several microseconds.  Returns false if the bounded wait gave up.
+// item back by several microseconds.  Returns false if the bounded wait gave up.  `rounds`: where the
+// warp's mbarrier is not re-initialised from item to item, the number of rounds it has been through.
 template <int D>
 struct TileUpdate {
     static constexpr int ROW_BYTES = D * 2;                       // one K or V row of one head
@@ -131,13 +132,14 @@ struct TileUpdate {
 
 template <int D>
 __device__ __forceinline__ bool tile_update_cache(const KernelArgs& a, const TileCtx& it, int w, int lane, uint32_t stage,
-                                                  uint32_t bar, volatile uint32_t* abort_flag, uint32_t* status) {
+                                                  uint32_t bar, volatile uint32_t* abort_flag, uint32_t* status,
+                                                  int* rounds = nullptr) {
     using U = TileUpdate<D>;
     constexpr int ROW = U::ROW_BYTES, TPW = U::TPW;
     const int ps = a.page_size;
     const int64_t slot_elems = (int64_t)2 * a.h_kv * D;
     const uint32_t mine = stage + w * U::WARP_BYTES + lane * 2 * ROW;
-    int round = 0;
+    int round = rounds ? *rounds : 0;
     for (int t0 = w * TPW; t0 < it.n_tok; t0 += 2 * TPW, ++round) {
         const int nt = min(TPW, it.n_tok - t0);
         const bool act = lane < nt;
@@ -166,6 +168,7 @@ __device__ __forceinline__ bool tile_update_cache(const KernelArgs& a, const Til
         }
         __syncwarp();
     }
+    if (rounds) *rounds = round;
     return true;
 }
 
