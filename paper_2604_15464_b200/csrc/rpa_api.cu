@@ -25,7 +25,7 @@ struct rpa_handle {
     Plan plan;
     int planned_num_seqs = -1;
     uint32_t ablation = 0;
-    int tile_pair_mode = 0;  // 0: two-tile kernel only; 1: host-planned steps run their tile items on the CTA-pair kernel
+    int tile_pair_mode = 2;  // tile items of host-made plans: 0 two-tile kernel, 1 CTA-pair kernel, 2 the pair kernel where every tile-routed sequence is long
     bool plan_pair = false;  // the current host-made plan's tile items are pair items
     std::string last_error;
 
@@ -223,6 +223,30 @@ void log_plan(const rpa_handle* h) {
             i.gpu_launches, i.algorithmic_bytes / 1e9, i.algorithmic_flops / 1e9, i.row_bytes / 1e9, i.tile_flops / 1e9);
 }
 
+// Do this batch's tile items run on the CTA-pair kernel?  It wants items of four full query tiles:
+// a shorter item leaves the pair's second CTA (or half of each CTA) without rows.  So, unless told
+// otherwise, it is chosen when every sequence the planner routes to the tile kernel brings at least
+// two full pair items of new tokens (long prefill and long chunks), and left alone for small-q steps
+// over long contexts and for short prompts (which the two-tile kernel splits by key blocks or packs).
+bool pair_kernel_wanted(const rpa_handle* h, const int32_t* cu_q_lens, const int32_t* kv_lens, int32_t num_seqs) {
+    const rpa_config_t& c = h->cfg;
+    const int h_g = c.num_q_heads / c.num_kv_heads;
+    if (h->tile_pair_mode == 0 || h->policy.tile_min_q <= 0 || c.kv_dtype != RPA_KV_BF16 || !tile2_kernel_supported(c.head_dim, h_g))
+        return false;
+    if (h->plan_only && h->tile_pair_mode != 1) return false;  // (no device: plan what every device can run)
+    if (h->tile_pair_mode == 1) return true;
+    if (!cu_q_lens || !kv_lens) return false;
+    const int64_t long_q = 2 * tile2_kernel_tokens(h_g);
+    bool any = false;
+    for (int32_t r = 0; r < num_seqs; ++r) {
+        const int64_t q = (int64_t)cu_q_lens[r + 1] - cu_q_lens[r];
+        if (!sequence_routed_to_tile(c, h->policy, q, kv_lens[r])) continue;
+        if (q < long_q) return false;
+        any = true;
+    }
+    return any;
+}
+
 // Events recorded outside a capture cannot be waited for inside one (and the other way round): while
 // a stream is being captured into a graph, the capture's own order stands in for the handle's events.
 bool stream_is_capturing(cudaStream_t s) {
@@ -349,7 +373,7 @@ rpa_status_t rpa_plan(rpa_handle_t* h, const int32_t* cu_q_lens_host, const int3
     if (!h) return RPA_ERR_INVALID_ARG;
     h->planned_num_seqs = -1;
     h->device_planned = false;
-    const bool pair = h->tile_pair_mode == 1 && h->policy.tile_min_q > 0;
+    const bool pair = pair_kernel_wanted(h, cu_q_lens_host, kv_lens_host, num_seqs);
     PlanPolicy pol = h->policy;
     if (pair) {  // pair items: twice the tokens, never packed
         pol.tile_tokens = tile2_kernel_tokens(h->cfg.num_q_heads / h->cfg.num_kv_heads);
@@ -918,9 +942,9 @@ rpa_status_t rpa_set_tile_min_q(rpa_handle_t* h, int32_t tokens) {
 }
 
 rpa_status_t rpa_set_tile_pair(rpa_handle_t* h, int32_t mode) {
-    if (!h || mode < 0 || mode > 1) return RPA_ERR_INVALID_ARG;
+    if (!h || mode < 0 || mode > 2) return RPA_ERR_INVALID_ARG;
     const int h_g = h->cfg.num_q_heads / h->cfg.num_kv_heads;
-    if (mode && (h->cfg.kv_dtype != RPA_KV_BF16 || !tile2_kernel_supported(h->cfg.head_dim, h_g))) return RPA_ERR_UNSUPPORTED;
+    if (mode == 1 && (h->cfg.kv_dtype != RPA_KV_BF16 || !tile2_kernel_supported(h->cfg.head_dim, h_g))) return RPA_ERR_UNSUPPORTED;
     h->tile_pair_mode = mode;
     h->plan.valid = false;
     h->planned_num_seqs = -1;

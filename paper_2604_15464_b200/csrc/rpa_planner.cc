@@ -43,6 +43,10 @@ inline bool routed_to_tile(const rpa_config_t& cfg, const PlanPolicy& policy, in
 
 }  // namespace
 
+bool sequence_routed_to_tile(const rpa_config_t& cfg, const PlanPolicy& policy, int64_t q_len, int64_t kv_len) {
+    return routed_to_tile(cfg, policy, q_len, kv_len);
+}
+
 rpa_status_t build_plan(const rpa_config_t& cfg, const PlanPolicy& policy, const int32_t* cu_q_lens,
                         const int32_t* kv_lens, int32_t num_seqs, Plan& plan) {
     plan.valid = false;

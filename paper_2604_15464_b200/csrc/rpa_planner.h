@@ -50,6 +50,9 @@ struct Plan {
     bool valid = false;
 };
 
+// Does the planner route a sequence of these lengths to the tile kernel?
+bool sequence_routed_to_tile(const rpa_config_t& cfg, const PlanPolicy& policy, int64_t q_len, int64_t kv_len);
+
 // Validates the lengths against `cfg` and fills `plan`.  No CUDA call.
 rpa_status_t build_plan(const rpa_config_t& cfg, const PlanPolicy& policy, const int32_t* cu_q_lens,
                         const int32_t* kv_lens, int32_t num_seqs, Plan& plan);

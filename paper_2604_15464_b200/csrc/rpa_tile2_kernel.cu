@@ -40,6 +40,10 @@
 #include "rpa_sm100.cuh"
 #include "rpa_tile_common.cuh"
 
+#ifndef RPA_PAIR_POLY
+#define RPA_PAIR_POLY 0
+#endif
+
 namespace rpa {
 
 using namespace sm100;
@@ -52,6 +56,7 @@ constexpr int kPairThreads = 384;  // 12 warps = 3 warpgroups per CTA
 constexpr int kPairWarps = 2 * (kPairThreads / 32);
 constexpr uint32_t kTmemCols = 512;
 constexpr float kRescaleThreshold = 8.f;  // log2 units
+constexpr int kBatchSpacing = 1360; // cycles between the product batches of the two tiles (see the MMA issuer)
 constexpr int kFetchAhead = 3;     // the next item is drawn when the running one has this many key blocks to go
 constexpr int D = 128;
 
@@ -355,6 +360,17 @@ rpa_tile2_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
         auto k_landed = [&](int f, uint32_t code) {  // fill f of the K ring, both halves
             return wait(BAR_KFULL + (f & 1), (f >> 1) & 1, code) && wait(BAR_KPEER + (f & 1), (f >> 1) & 1, code + 1);
         };
+        // The two tiles' softmax phases should not run at the same time: each runs at the special-
+        // function unit's full rate only when it has the unit to itself.  Nothing in the chain of
+        // dependencies sets the offset between the tiles, so the issuing warp does: a tile's batch of
+        // products (PV of this block, scores of the next) is not issued before `spacing` cycles have
+        // passed since the other tile's batch, which keeps the tiles about half a period apart.
+        const long long spacing = a.ablation >> 16 ? (long long)(a.ablation >> 16) * 16 : kBatchSpacing;
+        long long t_batch = clock64() - spacing;
+        auto keep_apart = [&]() {
+            while (clock64() - t_batch < spacing) {}
+            t_batch = clock64();
+        };
         int gb = 0;
         TileCtx it, nxt;
         int item, nxt_item = n_items;
@@ -367,6 +383,11 @@ rpa_tile2_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
                 if (elect_one()) {
                     issue_qk(0, 0, 0);
                     tc_commit_pair(bar(BAR_SFULL + 0));
+                }
+                __syncwarp();
+                keep_apart();
+                keep_apart();
+                if (elect_one()) {
                     issue_qk(0, 1, 0);
                     tc_commit_pair(bar(BAR_SFULL + 1));
                     tc_commit_pair(bar(BAR_KEMPTY + 0));
@@ -386,6 +407,7 @@ rpa_tile2_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
                     const bool last = j + 1 == n_blocks;
                     ok = wait(BAR_PREADY + 0, f & 1, 0x26);
                     if (!ok) break;
+                    keep_apart();
                     tc_fence_after();
                     if (elect_one()) {
                         issue_pv(0, st, j == 0);
@@ -415,6 +437,7 @@ rpa_tile2_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
                     }
                     ok = wait(BAR_PREADY + 1, f & 1, 0x27);
                     if (!ok) break;
+                    keep_apart();
                     tc_fence_after();
                     if (elect_one()) {
                         issue_pv(1, st, j == 0);
@@ -581,7 +604,8 @@ rpa_tile2_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
                 for (int i = 0; i < 32; ++i) {
                     float x0, x1;
                     fma2_bcast(x0, x1, s[ch * 64 + 2 * i], s[ch * 64 + 2 * i + 1], a.scale_log2, neg_m);
-                    const float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
+                    const bool poly = RPA_PAIR_POLY && (i & 3) == 3;
+                    const float p0 = poly ? poly_exp2(x0) : fast_exp2(x0), p1 = poly ? poly_exp2(x1) : fast_exp2(x1);
                     add2(lp[2 * (i & 3)], lp[2 * (i & 3) + 1], p0, p1);
                     p32[i] = pack_bf16x2(p0, p1);
                 }
