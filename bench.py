@@ -58,7 +58,7 @@ NOMINAL_BF16_TFLOPS = 2250.0
 # (keys: workload, dominant kernel, FP8 cache)
 NCU_TRAFFIC = {("decode", "row", False): (2.3820e9, "profiles/row_kernel_llama_decode.md"),
                ("decode", "row", True): (1.1994e9, "profiles/row_kernel_fp8_llama_decode.md"),
-               ("prefill", "tile", False): (0.7677e9, "profiles/tile_kernel_llama_prefill.md"),
+               ("prefill", "tile", False): (0.7675e9, "profiles/pair_kernel_llama_prefill.md"),
                ("mixed", "row", False): (3.3463e9, "profiles/mixed_llama_launch_list.md")}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
@@ -409,7 +409,8 @@ def run_leg(workload, args, rank, world, local, dist, peaks):
         else:  # the split-KV row kernel streams the cache: HBM
             achieved = info["row_bytes"] / 1e9 / (k_ms * 1e-3)
             peak, kbound, runit, nominal = float(peaks["hbm_gbs"]), "hbm", "GB/s", NOMINAL_HBM_GBS
-        r = {"bound": kbound, "kernel": f"rpa_{kind}_kernel", "achieved": achieved, "peak": peak, "unit": runit,
+        kname = {"tile": {2: "rpa_tile1_kernel", 3: "rpa_tile2_kernel"}.get(info.get("tile_kernel", 1), "rpa_tile_kernel")}.get(kind, f"rpa_{kind}_kernel")
+        r = {"bound": kbound, "kernel": kname, "achieved": achieved, "peak": peak, "unit": runit,
              "frac": achieved / peak, "peak_source": peaks["_source"], "traffic": None, "kernel_ms": k_ms,
              "kernel_launches": launches, "kernel_share_of_step": k_ms / max(1e-9, ms_per_step),
              "frac_of_nominal": achieved / nominal}

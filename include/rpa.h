@@ -121,6 +121,9 @@ typedef struct {
     int64_t workspace_bytes;    /* split-KV partials this plan uses                                  */
     int64_t row_bytes;          /* algorithmic bytes of the sequences served by the row kernel       */
     int64_t tile_flops;         /* algorithmic FLOPs of the sequences served by the tile kernel      */
+    int32_t tile_kernel;        /* which tensor-core kernel runs the tile items: 0 none, 1 two-tile,
+                                   2 single-tile (d_k = 256), 3 CTA pair (see rpa_set_tile_pair)       */
+    int32_t reserved;
 } rpa_plan_info_t;
 
 /*

@@ -215,10 +215,11 @@ void log_plan(const rpa_handle* h) {
     const rpa_plan_info_t& i = h->plan.info;
     fprintf(stderr,
             "[rpa] plan: %s batch, %d seqs (%d decode, %d prefill), %d new tokens; row kernel %d items (largest %d rows, "
-            "split chunk %d tokens, %d combine groups, %d partials), tile kernel %d items on %d CTAs; %d launches, %.3f GB, "
+            "split chunk %d tokens, %d combine groups, %d partials), %s kernel %d items on %d CTAs; %d launches, %.3f GB, "
             "%.3f GFLOP (row %.3f GB, tile %.3f GFLOP)\n",
             kCase[i.batch_case & 3], i.num_seqs, i.num_decode_seqs, i.num_prefill_seqs, i.num_tokens, i.num_row_items,
-            h->plan.row_rows_max, i.kv_chunk_tokens, i.num_combine_groups, h->plan.num_partials, i.num_tile_items,
+            h->plan.row_rows_max, i.kv_chunk_tokens, i.num_combine_groups, h->plan.num_partials,
+            i.tile_kernel == 3 ? "pair" : i.tile_kernel == 2 ? "single-tile" : "tile", i.num_tile_items,
             h->plan.tile_ctas > 0 ? h->plan.tile_ctas : (i.num_tile_items > 0 ? std::min(i.num_tile_items, h->num_sms) : 0),
             i.gpu_launches, i.algorithmic_bytes / 1e9, i.algorithmic_flops / 1e9, i.row_bytes / 1e9, i.tile_flops / 1e9);
 }
@@ -382,6 +383,9 @@ rpa_status_t rpa_plan(rpa_handle_t* h, const int32_t* cu_q_lens_host, const int3
     rpa_status_t st = build_plan(h->cfg, pol, cu_q_lens_host, kv_lens_host, num_seqs, h->plan);
     if (st != RPA_OK) return st;
     h->plan_pair = pair;
+    h->plan.info.tile_kernel = h->plan.tiles.empty() ? 0
+                               : pair ? 3
+                               : tile1_kernel_supported(h->cfg.head_dim, h->cfg.num_q_heads / h->cfg.num_kv_heads) ? 2 : 1;
     if (plan_log_enabled()) log_plan(h);
     if (!h->plan_only) {
         st = ensure_device(h);
