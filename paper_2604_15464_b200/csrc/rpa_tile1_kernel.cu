@@ -384,7 +384,7 @@ rpa_tile1_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
                     }
                 }
             } else if (!(a.ablation & kAblateUpdate) && (it.flags & kFlagWriteKv)) {
-                tile_update_cache<D>(a, it, warp - 2, lane, smem_base + C::OFF_UPD, bar(T1_UPD + warp - 2), abort_flag, a.status);
+                tile_update_cache<D>(a, it, warp - 2, lane, smem_base + C::OFF_UPD);
             }
             if (warp == 3 && !fetch_early) fetch_next();
         } else {

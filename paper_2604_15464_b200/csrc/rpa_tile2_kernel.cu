@@ -151,7 +151,7 @@ rpa_tile2_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
     // drawing warp has published it, reads it, and tells the drawing warp that this warp is done with
     // the slot.  Returns false when the wait gave up.
     auto take_item = [&](int n, TileCtx& it, int& item) -> bool {
-        const bool ok = mbar_wait_pair<true>(bar(BAR_ITEM + (n & 1)), (n >> 1) & 1, abort_flag, peer_abort, a.status, 0x60);
+        const bool ok = wait(BAR_ITEM + (n & 1), (n >> 1) & 1, 0x60);
         if (!__all_sync(0xffffffffu, ok)) return false;
         const volatile int* slot = item_slots + (n & 1) * RAW_INTS;
         item = slot[RAW_ITEM];
@@ -469,16 +469,19 @@ rpa_tile2_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
             draw_and_fetch_tile(a, true, fallback, slot, lane);
             __syncwarp();
             if (lane == 0) {
-                const uint32_t dst = map_to_cta(smem_u32(const_cast<int*>(slot)), 1u);
-                for (int k = 0; k < RAW_BOUNDS + 2; ++k) st_cluster_u32(dst + 4u * k, (uint32_t)slot[k]);
+                // the second CTA gets its copy from the copy engine, which counts the bytes at that CTA's
+                // barrier (a releasing arrival across the pair costs as much as a device-wide fence)
+                const uint32_t src = smem_u32(const_cast<int*>(slot)), remote_bar = map_to_cta(bar(BAR_ITEM + (n & 1)), 1u);
+                fence_proxy_async_smem();
+                mbar_arrive_expect_tx_cluster(remote_bar, RAW_INTS * 4);
+                bulk_copy_to_cta(map_to_cta(src, 1u), src, RAW_INTS * 4, remote_bar);
                 mbar_arrive(bar(BAR_ITEM + (n & 1)));
-                mbar_arrive_cluster_release(map_to_cta(bar(BAR_ITEM + (n & 1)), 1u));  // the entry written above is visible to its waiters
             }
             __syncwarp();
             return true;
         };
         const bool drawer = warp == 3 && first_cta;
-        int gb = 0, upd_rounds = 0;
+        int gb = 0;
         bool ok = true;
         if (drawer) ok = publish(0, 0);
         for (int n = 0; ok; ++n) {
@@ -491,8 +494,7 @@ rpa_tile2_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
                 TileCtx own = it;
                 own.q_tok0 = it.q_tok0 + (int)rank * 2 * TQ;
                 own.n_tok = own_tokens(it);
-                ok = tile_update_cache<D>(a, own, warp - 2, lane, smem_base + C::OFF_UPD, bar(BAR_UPD + warp - 2), abort_flag, a.status,
-                                          &upd_rounds);
+                tile_update_cache<D>(a, own, warp - 2, lane, smem_base + C::OFF_UPD);
             }
             if (drawer && ok) {
                 if (lane == 0) {

@@ -115,61 +115,104 @@ __device__ __forceinline__ int packed_seq_of(const TileCtx& it, int tok) {
     return lo;
 }
 
-// Fused cache update of one item by two warps (`w` = 0 or 1): K and V rows of the item's own tokens
-// for its KV head, moved by the bulk-copy engine.  A lane owns one token per round: it fetches the
-// token's K row and V row into the warp's staging area (completion on the warp's mbarrier `bar`),
-// then writes both with one bulk store, since K_h and V_h are neighbours in a cache slot.  Plain
-// loads and stores would queue behind the epilogue's stores in the load/store unit and hold a short
-// item back by several microseconds.  Returns false if the bounded wait gave up.  `rounds`: where the
-// warp's mbarrier is not re-initialised from item to item, the number of rounds it has been through.
+// Fused cache update of an item ("Update U_kv" of Algorithm 1): the K and V rows of the item's own
+// tokens for its KV head go into their cache slots, a round of TPW tokens at a time.  The rows of a
+// round are fetched into shared memory with 16-byte asynchronous copies (one instruction moves 512
+// bytes for the warp and does not block it), then written out with 16-byte stores, 512 contiguous
+// bytes per token at d_k = 128 since K_h and V_h are neighbours in a slot.  (An earlier version gave
+// each lane a token and moved its rows with per-thread bulk copies: the copy engine takes such
+// copies one thread at a time, about 60 cycles each - 192 of them per 64 tokens, which is what an
+// item of a short prompt then cost.)  A lane computes the slot of "its" token of the round (token =
+// lane) and the others read it by shuffle; a lane stores exactly the bytes it fetched, so nothing
+// but its own wait orders the two.  BUFS: staging buffers of WARP_BYTES each; with two, the next
+// round's rows travel while this round's are written.
 template <int D>
 struct TileUpdate {
     static constexpr int ROW_BYTES = D * 2;                       // one K or V row of one head
-    static constexpr int TPW = 8192 / ROW_BYTES < 32 ? 8192 / ROW_BYTES : 32;  // tokens per warp and round
+    static constexpr int TPW = 8192 / ROW_BYTES < 32 ? 8192 / ROW_BYTES : 32;  // tokens per round
     static constexpr int WARP_BYTES = TPW * 2 * ROW_BYTES;
     static constexpr int STAGE_BYTES = 2 * WARP_BYTES;
 };
 
-template <int D>
-__device__ __forceinline__ bool tile_update_cache(const KernelArgs& a, const TileCtx& it, int w, int lane, uint32_t stage,
-                                                  uint32_t bar, volatile uint32_t* abort_flag, uint32_t* status,
-                                                  int* rounds = nullptr) {
+__device__ __forceinline__ void st_global_v4(void* p, const uint4& v) {
+    asm volatile("st.global.v4.u32 [%0], {%1,%2,%3,%4};\n" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+
+// Rounds t_first, t_first + t_step, ... (token offsets inside the item) by one warp.  The warps of
+// the first warpgroup get an issue slot every few cycles only (the softmax warps own the schedulers),
+// so the loops below are kept to a handful of instructions per 512 bytes moved.
+template <int D, int BUFS>
+__device__ __forceinline__ void tile_update_rounds(const KernelArgs& a, const TileCtx& it, int t_first, int t_step, int lane, uint32_t stage) {
     using U = TileUpdate<D>;
-    constexpr int ROW = U::ROW_BYTES, TPW = U::TPW;
+    constexpr int ROW = U::ROW_BYTES, TPW = U::TPW, CPT = 2 * ROW / 16, HALF = CPT / 2;  // 16-byte pieces per token: K row, then V row
+    constexpr int STEPS = TPW * CPT / 32;                                                // warp-wide instructions per full round
+    static_assert(BUFS == 1 || BUFS == 2, "one or two staging buffers");
+    static_assert((CPT & (CPT - 1)) == 0 && TPW * CPT % 32 == 0, "pieces per token: a power of two");
     const int ps = a.page_size;
-    const int64_t slot_elems = (int64_t)2 * a.h_kv * D;
-    const uint32_t mine = stage + w * U::WARP_BYTES + lane * 2 * ROW;
-    int round = rounds ? *rounds : 0;
-    for (int t0 = w * TPW; t0 < it.n_tok; t0 += 2 * TPW, ++round) {
-        const int nt = min(TPW, it.n_tok - t0);
-        const bool act = lane < nt;
-        const int tok = it.q_tok0 + t0 + lane;
-        int pos = it.c + tok;
-        const int32_t* pt_row = it.pt_row;
-        if (it.n_seqs > 1 && act) {  // packed item: the token's own sequence, page-table row and position
-            const int k = packed_seq_of(it, tok);
-            pos = tok - it.bounds[k];
-            pt_row += (int64_t)k * a.max_pages_per_seq;
+    uint8_t* cache = reinterpret_cast<uint8_t*>(a.kv_cache);
+    const int64_t tok_stride = (int64_t)a.h_kv * D;  // elements from one token's row to the next
+    // writes a landed round out of its buffer; slot: this lane's token's cache slot in units of ROW
+    // bytes (~0: none), read by the other lanes
+    auto write_out = [&](uint32_t buf, int nt, uint32_t slot) {
+#pragma unroll 4
+        for (int s = 0; s < STEPS; ++s) {
+            const int idx = s * 32 + lane, t = idx / CPT, piece = idx % CPT;
+            const uint32_t slot_t = __shfl_sync(0xffffffffu, slot, t);
+            if (t < nt && slot_t != ~0u) st_global_v4(cache + (int64_t)slot_t * ROW + piece * 16, ld_shared_v4(buf + idx * 16));
         }
-        const int page = act ? pt_row[pos / ps] : 0;
-        const bool store_ok = act && debug_write_page_ok(a, page);  // (always true outside the bounds-checked build)
-        if (lane == 0) sm100::mbar_arrive_expect_tx(bar, (uint32_t)nt * 2 * ROW);
-        __syncwarp();
-        if (act) {
-            const int64_t src = (((int64_t)it.cu + tok) * a.h_kv + it.h) * D;
-            sm100::bulk_load(mine, a.new_k + src, ROW, bar);
-            sm100::bulk_load(mine + ROW, a.new_v + src, ROW, bar);
+    };
+    int r = 0, prev_nt = 0;
+    uint32_t prev_slot = ~0u;
+    for (int t0 = t_first;; t0 += t_step, ++r) {
+        const bool have = t0 < it.n_tok;
+        const uint32_t buf = stage + (r % BUFS) * U::WARP_BYTES;
+        int nt = 0;
+        uint32_t slot = ~0u;
+        if (have) {
+            nt = min(TPW, it.n_tok - t0);
+            const bool act = lane < nt;
+            const int tok = it.q_tok0 + t0 + lane;
+            int pos = it.c + tok;
+            const int32_t* pt_row = it.pt_row;
+            if (it.n_seqs > 1 && act) {  // packed item: the token's own sequence, page-table row and position
+                const int k = packed_seq_of(it, tok);
+                pos = tok - it.bounds[k];
+                pt_row += (int64_t)k * a.max_pages_per_seq;
+            }
+            const int page = act ? pt_row[pos / ps] : 0;
+            if (act && debug_write_page_ok(a, page))  // (always true for a token of the round outside the bounds-checked build)
+                slot = (uint32_t)(((int64_t)page * ps + pos % ps) * 2 * a.h_kv + 2 * it.h);
+            const uint16_t* row0 = a.new_k + (((int64_t)it.cu + it.q_tok0 + t0) * a.h_kv + it.h) * D;  // token 0 of the round, K
+            const int64_t v_minus_k = a.new_v - a.new_k;
+#pragma unroll 4
+            for (int s = 0; s < STEPS; ++s) {
+                const int idx = s * 32 + lane, t = idx / CPT, piece = idx % CPT;
+                const uint16_t* src = row0 + t * tok_stride + (piece % HALF) * 8 + (piece < HALF ? 0 : v_minus_k);
+                if (t < nt) cp_async_16(buf + idx * 16, src, 16);
+            }
+            cp_async_commit();
         }
-        if (!sm100::mbar_wait(bar, round & 1, abort_flag, status, 0x40 + w)) return false;
-        if (store_ok) {
-            sm100::bulk_store(a.kv_cache + ((int64_t)page * ps + pos % ps) * slot_elems + (int64_t)2 * it.h * D, mine, 2 * ROW);
-            sm100::bulk_commit();
-            sm100::bulk_wait_read();  // the staging area is free again
+        if (BUFS == 1) {
+            if (!have) break;
+            cp_async_wait<0>();
+            write_out(buf, nt, slot);
+        } else {
+            if (prev_nt > 0) {  // the round before has landed (all but the group just committed are complete)
+                if (have) cp_async_wait<1>(); else cp_async_wait<0>();
+                write_out(stage + ((r - 1) % BUFS) * U::WARP_BYTES, prev_nt, prev_slot);
+            }
+            if (!have) break;
+            prev_nt = nt, prev_slot = slot;
         }
-        __syncwarp();
     }
-    if (rounds) *rounds = round;
-    return true;
+}
+
+// The update of one item shared by two warps (`w` = 0 or 1), each with its own staging buffer at
+// stage + w * WARP_BYTES: warp w takes every other round.
+template <int D>
+__device__ __forceinline__ void tile_update_cache(const KernelArgs& a, const TileCtx& it, int w, int lane, uint32_t stage) {
+    using U = TileUpdate<D>;
+    tile_update_rounds<D, 1>(a, it, w * U::TPW, 2 * U::TPW, lane, stage + w * U::WARP_BYTES);
 }
 
 // FP8 cache: the pass that runs before the tile kernel.  One CTA per tile item quantises the
