@@ -52,11 +52,12 @@ namespace {
 
 constexpr int kBlockN = 128;       // KV positions per block
 constexpr int kHalfN = 64;         // ... of which each CTA of the pair stages this many keys
+constexpr int kBoxN = 32;          // ... as two runs of 32: keys [32r, 32r+32) and [64+32r, 64+32r+32) for CTA r (see the MMA issuer)
 constexpr int kPairThreads = 384;  // 12 warps = 3 warpgroups per CTA
 constexpr int kPairWarps = 2 * (kPairThreads / 32);
 constexpr uint32_t kTmemCols = 512;
 constexpr float kRescaleThreshold = 8.f;  // log2 units
-constexpr int kBatchSpacing = 1360; // cycles between the product batches of the two tiles (see the MMA issuer)
+constexpr int kBatchSpacing = 1040; // cycles between the product batches of the two tiles (see the MMA issuer)
 constexpr int kFetchAhead = 3;     // the next item is drawn when the running one has this many key blocks to go
 constexpr int D = 128;
 
@@ -80,9 +81,9 @@ struct PairCfg {
 };
 
 // barrier slots (8 bytes each), two of each kind.  Every CTA has all of them at the same offsets;
-// QPEER/KPEER/VPEER, PREADY and ITEMFREE are used in the first CTA only.
+// QPEER/KPEER/VPEER, PREADY, SCONS and ITEMFREE are used in the first CTA only.
 enum { BAR_Q = 0, BAR_QPEER = 2, BAR_QFREE = 4, BAR_KFULL = 6, BAR_KEMPTY = 8, BAR_VFULL = 10, BAR_VEMPTY = 12, BAR_KPEER = 14,
-       BAR_VPEER = 16, BAR_SFULL = 18, BAR_PREADY = 20, BAR_ODONE = 22, BAR_UPD = 24, BAR_EPI = 26, BAR_ITEM = 28,
+       BAR_VPEER = 16, BAR_SFULL = 18, BAR_PREADY = 20, BAR_ODONE = 22, BAR_SCONS = 24, BAR_EPI = 26, BAR_ITEM = 28,
        BAR_ITEMFREE = 30, BAR_COUNT = 32 };
 static_assert(8 * BAR_COUNT <= 256, "barrier block");
 
@@ -129,7 +130,7 @@ rpa_tile2_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
             mbar_init(bar(BAR_SFULL + s), 1);
             mbar_init(bar(BAR_PREADY + s), 8);  // one arrival per softmax warp of the tile, both CTAs
             mbar_init(bar(BAR_ODONE + s), 1);
-            mbar_init(bar(BAR_UPD + s), 1);
+            mbar_init(bar(BAR_SCONS + s), 8);   // the tile's softmax warps of both CTAs have taken S into registers
             mbar_init(bar(BAR_EPI + s), 128);
             mbar_init(bar(BAR_ITEM + s), 1);
             mbar_init(bar(BAR_ITEMFREE + s), kPairWarps);  // every warp of both CTAs has read the slot
@@ -190,7 +191,7 @@ rpa_tile2_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
             prefetch_tmap(&maps.new_k);
             prefetch_tmap(&maps.new_v);
         }
-        const int box_rows = page_box_rows(ps, kHalfN);
+        const int box_rows = page_box_rows(ps, kBoxN);
         int gb = 0;  // key blocks of earlier items: block j of the running item is fill gb + j of either ring
         bool ok = true;
         for (int n = 0; ok; ++n) {
@@ -226,12 +227,15 @@ rpa_tile2_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
                 const int f = gb + j, st = f & 1;
                 if (!debug_stage_ok(a, st, C::KS)) return false;
                 const int rows = kv ? kBlockN : kHalfN;            // rows of the block this CTA stages
-                const int row0 = kv ? 0 : (int)rank * kHalfN;      // ... starting at this row of the block
                 const int boxes = rows / box_rows;
+                // row of the block that lands in row lr of the stage: V takes the block as it is; the keys of
+                // CTA r are the runs [32r, 32r + 32) and [64 + 32r, 64 + 32r + 32)
+                const int lr = lane * box_rows;
+                const int blk_row = kv ? lr : (lr / kBoxN) * kHalfN + (int)rank * kBoxN + lr % kBoxN;
                 int page = 0, slot0 = 0;
                 bool sub_valid = false;
                 if (ctx) {
-                    const int pos = j * kBlockN + row0 + lane * box_rows;
+                    const int pos = j * kBlockN + blk_row;
                     sub_valid = lane < boxes && pos < c;
                     if (sub_valid) {
                         page = debug_read_page(a, pt_row[pos / ps]);
@@ -267,12 +271,15 @@ rpa_tile2_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
                     const int new_row0 = cu + (j - n_ctx_blocks) * kBlockN;
                     if (kv) {
 #pragma unroll
-                        for (int i = 0; i < kBlockN / kHalfN; ++i)
-                            tma_load_3d(dst + i * C::HALF_BLK, &maps.new_v, (int)rank * 64, h, new_row0 + i * kHalfN, bar(full));
+                        for (int i = 0; i < kBlockN / kBoxN; ++i)
+                            tma_load_3d(dst + i * kBoxN * 128, &maps.new_v, (int)rank * 64, h, new_row0 + i * kBoxN, bar(full));
                     } else {
 #pragma unroll
                         for (int b = 0; b < C::NBLK; ++b)
-                            tma_load_3d(dst + b * C::HALF_BLK, &maps.new_k, b * 64, h, new_row0 + (int)rank * kHalfN, bar(full));
+#pragma unroll
+                            for (int run = 0; run < 2; ++run)
+                                tma_load_3d(dst + b * C::HALF_BLK + run * kBoxN * 128, &maps.new_k, b * 64, h,
+                                            new_row0 + run * kHalfN + (int)rank * kBoxN, bar(full));
                     }
                 }
                 return true;
@@ -329,22 +336,29 @@ rpa_tile2_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
         }
       } else if (warp == 1) {
         // ================================ MMA issuer (first CTA, for the pair) ================================
-        constexpr uint32_t idesc_qk = instr_desc_bf16(256, kBlockN, 0, 0);
+        constexpr uint32_t idesc_qk = instr_desc_bf16(256, kBlockN / 2, 0, 0);
         constexpr uint32_t idesc_pv = instr_desc_bf16(256, D, 0, 1);
         constexpr uint32_t desc_hi = smem_desc_sw128_hi(1024);
         const uint32_t k_lo = smem_desc_sw128_lo(smem_base + C::OFF_K, 16);
         const uint32_t v_lo = smem_desc_sw128_lo(smem_base + C::OFF_V, C::BLK_BYTES);
         const bool no_compute = a.ablation & kAblateCompute;  // bench switch: commits without products
-        // S_x = Q_x K^T over d_k in steps of 16, tile x of both CTAs; the queries of item n, the keys in stage st
-        auto issue_qk = [&](int n, int x, int st) {
+        // The scores of a block are made by two products of 64 keys each: columns [0, 64) of S ("low":
+        // keys 0..63 of the block - run 0 of both CTAs' stages) and columns [64, 128) ("high").  The
+        // probabilities of block j go into the HIGH columns, so the low product of block j+1 does not
+        // have to wait for P_j V_j: it is issued as soon as the softmax warps have taken S_j into their
+        // registers, and runs while they work; only the high product stands behind P_j V_j in the
+        // tile's chain of dependencies (P ready -> PV -> scores -> softmax), 8 products of 64 keys
+        // instead of 8 of 128.
+        // S_x[:, 64 half ..] = Q_x K^T over d_k in steps of 16, tile x of both CTAs; queries of item n, keys in stage st
+        auto issue_qk = [&](int n, int x, int st, int half) {
             if (no_compute) return;
             const uint32_t ql = smem_desc_sw128_lo(smem_base + C::OFF_Q + ((n & 1) * 2 + x) * C::TILE_BYTES, 16);
-            const uint32_t kl = k_lo + st * (C::K_STAGE >> 4);
+            const uint32_t kl = k_lo + ((st * C::K_STAGE + half * kBoxN * 128) >> 4);
 #pragma unroll
             for (int ks = 0; ks < D / 16; ++ks) {
                 const uint32_t q_off = ((ks / 4) * C::BLK_BYTES + (ks % 4) * 32) >> 4;
                 const uint32_t k_off = ((ks / 4) * C::HALF_BLK + (ks % 4) * 32) >> 4;
-                umma_ss_pair(tm_s[x], make_desc(ql + q_off, desc_hi), make_desc(kl + k_off, desc_hi), idesc_qk, ks > 0);
+                umma_ss_pair(tm_s[x] + half * 64, make_desc(ql + q_off, desc_hi), make_desc(kl + k_off, desc_hi), idesc_qk, ks > 0);
             }
         };
         auto issue_pv = [&](int x, int st, bool first) {  // O_x (+)= P_x V over 128 positions in steps of 16
@@ -352,7 +366,7 @@ rpa_tile2_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
             const uint32_t vl = v_lo + st * (C::V_STAGE >> 4);
 #pragma unroll
             for (int kk = 0; kk < kBlockN / 16; ++kk)
-                umma_ts_pair(tm_o[x], tm_s[x] + kk * 8, make_desc(vl + kk * (2048 >> 4), desc_hi), idesc_pv, !(first && kk == 0));
+                umma_ts_pair(tm_o[x], tm_s[x] + 64 + kk * 8, make_desc(vl + kk * (2048 >> 4), desc_hi), idesc_pv, !(first && kk == 0));
         };
         auto q_landed = [&](int n) {
             return wait(BAR_Q + (n & 1), (n >> 1) & 1, 0x20) && wait(BAR_QPEER + (n & 1), (n >> 1) & 1, 0x21);
@@ -381,14 +395,16 @@ rpa_tile2_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
             if (ok) {
                 tc_fence_after();
                 if (elect_one()) {
-                    issue_qk(0, 0, 0);
+                    issue_qk(0, 0, 0, 0);
+                    issue_qk(0, 0, 0, 1);
                     tc_commit_pair(bar(BAR_SFULL + 0));
                 }
                 __syncwarp();
                 keep_apart();
                 keep_apart();
                 if (elect_one()) {
-                    issue_qk(0, 1, 0);
+                    issue_qk(0, 1, 0, 0);
+                    issue_qk(0, 1, 0, 1);
                     tc_commit_pair(bar(BAR_SFULL + 1));
                     tc_commit_pair(bar(BAR_KEMPTY + 0));
                 }
@@ -405,6 +421,23 @@ rpa_tile2_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
                     ok = wait(BAR_VPEER + st, ph, 0x25);
                     if (!ok) break;
                     const bool last = j + 1 == n_blocks;
+                    if (last && !looked) {  // what follows this item?  (drawn by now: the drawing warp watches `progress`)
+                        looked = true;
+                        ok = take_item(n + 1, nxt, nxt_item);
+                        if (!ok) break;
+                        have_next = nxt_item < n_items && debug_rows_ok(a, (long long)nxt.cu + nxt.q_tok0, nxt.n_tok);
+                    }
+                    // the next score products: the item's next block, or the next item's first one
+                    const bool more = !last || have_next;
+                    const int f1 = f + 1, st1 = f1 & 1, n1 = last ? n + 1 : n;
+                    if (more) {  // low half of tile A's next scores: S_A of this block is in the softmax warps' registers
+                        if (last) ok = q_landed(n + 1);
+                        ok = ok && k_landed(f1, 0x2C) && wait(BAR_SCONS + 0, f & 1, 0x2E);
+                        if (!ok) break;
+                        tc_fence_after();
+                        if (elect_one()) issue_qk(n1, 0, st1, 0);
+                        __syncwarp();
+                    }
                     ok = wait(BAR_PREADY + 0, f & 1, 0x26);
                     if (!ok) break;
                     keep_apart();
@@ -413,26 +446,17 @@ rpa_tile2_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
                         issue_pv(0, st, j == 0);
                         tc_commit_pair(bar(BAR_ODONE + 0));
                         *progress = f + 1;
-                    }
-                    __syncwarp();
-                    if (last && !looked) {  // what follows this item?  (drawn by now: the drawing warp watches `progress`)
-                        looked = true;
-                        ok = take_item(n + 1, nxt, nxt_item);
-                        if (!ok) break;
-                        have_next = nxt_item < n_items && debug_rows_ok(a, (long long)nxt.cu + nxt.q_tok0, nxt.n_tok);
-                    }
-                    // the next score product of tile A: the item's next block, or the next item's first one
-                    const bool more = !last || have_next;
-                    const int f1 = f + 1, st1 = f1 & 1, n1 = last ? n + 1 : n;
-                    if (more) {
-                        if (last) ok = q_landed(n + 1);
-                        ok = ok && k_landed(f1, 0x2C);
-                        if (!ok) break;
-                        tc_fence_after();
-                        if (elect_one()) {
-                            issue_qk(n1, 0, st1);
+                        if (more) {
+                            issue_qk(n1, 0, st1, 1);
                             tc_commit_pair(bar(BAR_SFULL + 0));
                         }
+                    }
+                    __syncwarp();
+                    if (more) {  // low half of tile B's next scores
+                        ok = wait(BAR_SCONS + 1, f & 1, 0x2F);
+                        if (!ok) break;
+                        tc_fence_after();
+                        if (elect_one()) issue_qk(n1, 1, st1, 0);
                         __syncwarp();
                     }
                     ok = wait(BAR_PREADY + 1, f & 1, 0x27);
@@ -444,7 +468,7 @@ rpa_tile2_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
                         tc_commit_pair(bar(BAR_ODONE + 1));
                         tc_commit_pair(bar(BAR_VEMPTY + st));
                         if (more) {
-                            issue_qk(n1, 1, st1);
+                            issue_qk(n1, 1, st1, 1);
                             tc_commit_pair(bar(BAR_SFULL + 1));
                             tc_commit_pair(bar(BAR_KEMPTY + st1));
                         }
@@ -518,6 +542,7 @@ rpa_tile2_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
         const uint32_t lane_sel = (uint32_t)(quarter * 32) << 16;
         const uint32_t s_addr = tm_s[x] + lane_sel, o_addr = tm_o[x] + lane_sel;
         const uint32_t pready = first_cta ? bar(BAR_PREADY + x) : first_cta_bar(BAR_PREADY + x);
+        const uint32_t scons = first_cta ? bar(BAR_SCONS + x) : first_cta_bar(BAR_SCONS + x);
         int gb = 0, epi_uses = 0;
         bool ok = true;
         for (int n = 0; ok; ++n) {
@@ -542,7 +567,10 @@ rpa_tile2_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
             if (a.ablation & kAblateCompute) {  // bench switch: hand over at once
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive_cluster(pready);
+                if (lane == 0) {
+                    mbar_arrive_cluster(scons);
+                    mbar_arrive_cluster(pready);
+                }
                 continue;
             }
             float s[kBlockN];
@@ -554,6 +582,9 @@ rpa_tile2_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
                 for (int i = 0; i < 32; ++i) s[ch * 32 + i] = __uint_as_float(r32[i]);
             }
             tc_wait_ld();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(scons);  // the low columns of S may be overwritten with the next block's scores
             // visible keys of this row inside the block: positions pos_base .. pos_base + n_vis - 1
             const bool ctx = j < n_ctx_blocks;
             const int pos_base = ctx ? j * kBlockN : c + (j - n_ctx_blocks) * kBlockN;
@@ -611,7 +642,7 @@ rpa_tile2_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
                     add2(lp[2 * (i & 3)], lp[2 * (i & 3) + 1], p0, p1);
                     p32[i] = pack_bf16x2(p0, p1);
                 }
-                tmem_st32(s_addr + ch * 32, p32);
+                tmem_st32(s_addr + 64 + ch * 32, p32);  // (the high columns: see the MMA issuer)
             }
             l_sum += ((lp[0] + lp[1]) + (lp[2] + lp[3])) + ((lp[4] + lp[5]) + (lp[6] + lp[7]));
             tc_wait_st();
@@ -742,7 +773,7 @@ int resident_pairs() {
 template <int G>
 cudaError_t launch_tile2(const KernelArgs& a, int64_t token_rows, TileMapCache* cache, cudaStream_t stream) {
     TileMaps maps;
-    if (!cached_tile_maps(cache, a, token_rows, D, G, 128 / G, kHalfN, &maps)) return cudaErrorInvalidValue;
+    if (!cached_tile_maps(cache, a, token_rows, D, G, 128 / G, kBoxN, &maps)) return cudaErrorInvalidValue;
     int pairs = resident_pairs<G>();
     if (a.num_tile_ctas > 0) pairs = min(pairs, max(1, a.num_tile_ctas / 2));
     pairs = min(pairs, a.num_tile_items);

@@ -88,9 +88,9 @@ def test_pair_kernel_two_calls_on_one_handle_and_back_to_the_two_tile_kernel():
 
 
 def test_pair_kernel_is_chosen_for_long_prefill_only():
-    # default mode: the pair kernel (items of 4 query tiles = 128 tokens at h_g = 4) when every sequence on the
-    # tile path has at least 256 new tokens; one shorter sequence keeps the batch on the two-tile kernel
-    for ql, kl, per_item in (([600, 300], [600, 1300], 128), ([600, 40], [600, 1300], 64), ([600, 300, 1], [600, 300, 900], 128)):
+    # default mode: the pair kernel (items of 4 query tiles = 128 tokens at h_g = 4) when every sequence of the
+    # batch has at least 256 new tokens; a shorter sequence or a decode row keeps the batch on the two-tile kernel
+    for ql, kl, per_item in (([600, 300], [600, 1300], 128), ([600, 40], [600, 1300], 64), ([600, 300, 1], [600, 300, 900], 64)):
         meta = wl.build_meta("pair_auto", ql, kl, num_q_heads=32, num_kv_heads=8, head_dim=128, page_size=16, seed=37)
         rapi = binding.Rpa.for_meta(meta)
         _, info = hz.full_parity(wl.materialize(meta, _dev()), rapi=rapi)
