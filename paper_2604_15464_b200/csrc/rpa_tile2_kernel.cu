@@ -514,13 +514,17 @@ rpa_tile2_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
             ok = take_item(n, it, item);
             if (!ok || item >= n_items) break;
             if (!debug_rows_ok(a, (long long)it.cu + it.q_tok0, it.n_tok)) break;
-            if (!(a.ablation & kAblateUpdate) && (it.flags & kFlagWriteKv)) {
+            // a short item's successor is drawn before this warp's share of the update (which takes longer
+            // than such an item runs), a long item's once it is within a few blocks of its end
+            const bool draw_first = it.n_blocks <= kFetchAhead;
+            if (drawer && draw_first) ok = publish(n + 1, n_items);
+            if (ok && !(a.ablation & kAblateUpdate) && (it.flags & kFlagWriteKv)) {
                 TileCtx own = it;
                 own.q_tok0 = it.q_tok0 + (int)rank * 2 * TQ;
                 own.n_tok = own_tokens(it);
                 tile_update_cache<D>(a, own, warp - 2, lane, smem_base + C::OFF_UPD);
             }
-            if (drawer && ok) {
+            if (drawer && ok && !draw_first) {
                 if (lane == 0) {
                     const long long t0 = clock64();
                     while (*progress < gb + it.n_blocks - kFetchAhead && !*abort_flag && clock64() - t0 < 4000000000LL) __nanosleep(256);
