@@ -58,7 +58,7 @@ NOMINAL_BF16_TFLOPS = 2250.0
 # (keys: workload, dominant kernel, FP8 cache)
 NCU_TRAFFIC = {("decode", "row", False): (2.3820e9, "profiles/row_kernel_llama_decode.md"),
                ("decode", "row", True): (1.1994e9, "profiles/row_kernel_fp8_llama_decode.md"),
-               ("prefill", "tile", False): (0.7675e9, "profiles/pair_kernel_llama_prefill.md"),
+               ("prefill", "tile", False): (0.7680e9, "profiles/pair_kernel_llama_prefill.md"),
                ("mixed", "row", False): (3.3463e9, "profiles/mixed_llama_launch_list.md")}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
