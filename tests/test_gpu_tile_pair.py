@@ -122,3 +122,53 @@ def test_pair_kernel_on_the_llama_prefill_workload_sampled_rows():
     (mx, mean), info = hz.sampled_parity(batch, seqs=[1, 2], rows_per_seq=192, whole_cache=True, rapi=rapi)
     assert info["batch_case_name"] == "prefill" and info["num_tile_items"] == 4 * 8 * 64
     rapi.close()
+
+
+def test_pair_kernel_in_the_bounds_checked_build():
+    """Good input: same results, nothing reported.  An out-of-range page id (one that still lies inside the
+    real allocation) in a context page and in a page that receives new tokens: named in the status word,
+    the read redirected to page 0, the write dropped."""
+    import dataclasses
+
+    from paper_2604_15464_b200 import build
+    debug_lib = build.build(debug=True)
+    tight = wl.build_meta("pair_dbg", [300, 260], [900, 260], num_q_heads=32, num_kv_heads=8, head_dim=128, page_size=16, seed=39,
+                          pool_slack=1.0)
+    rapi = binding.Rpa.for_meta(tight, library_path=debug_lib)
+    _, info = hz.full_parity(wl.materialize(tight, _dev(), canaries=True), rapi=rapi)
+    assert info["tile_kernel"] == 3 and rapi.rpa_poll_status() == 0
+    meta = dataclasses.replace(tight, num_pages=tight.num_pages + 8)  # the tensor holds 8 pages more than the handle knows of
+    batch = wl.materialize(meta, _dev())
+    bad = tight.num_pages + 5
+    tail_before = wl.bf16_bits(batch.kv_cache[tight.num_pages:]).copy()
+    out = torch.zeros_like(batch.q)
+    rapi.rpa_plan(meta.cu_q_lens, meta.kv_lens)
+    for seq, page_slot in ((0, 3), (1, (260 - 1) // 16)):  # a context page; the page of the last new tokens
+        table = batch.page_table.clone()
+        table[seq, page_slot] = bad
+        rapi.rpa_forward(batch.q, batch.new_k, batch.new_v, batch.kv_cache, table, batch.cu_q_lens, batch.kv_lens, out)
+        torch.cuda.synchronize()
+        word = rapi.rpa_poll_status()
+        assert word & (1 << 27) and (word >> 24) & 7 == 1 and (word & 0xFFFFFF) == bad
+        assert np.array_equal(tail_before, wl.bf16_bits(batch.kv_cache[tight.num_pages:]))  # nothing went through the bad id
+    hz.full_parity(wl.materialize(tight, _dev()), rapi=rapi)  # the handle keeps working
+    rapi.close()
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_pair_kernel_random_long_prefill_batches(seed):
+    """Seeded random pure-prefill batches (ragged lengths from 256 tokens up, with and without cached context,
+    several head groupings and page sizes): whole-batch parity, automatic choice of the pair kernel."""
+    rng = np.random.default_rng(4000 + seed)
+    hq, hkv = [(32, 8), (16, 2), (8, 8), (32, 4), (16, 16), (64, 8)][seed % 6]
+    tq4 = 4 * (128 // (hq // hkv))
+    n = int(rng.integers(1, 5))
+    ql = [int(rng.integers(2 * tq4, 2 * tq4 + 900)) for _ in range(n)]
+    kl = [q + (int(rng.integers(0, 1500)) if rng.integers(0, 2) else 0) for q in ql]
+    meta = wl.build_meta(f"pair_rand{seed}", ql, kl, num_q_heads=hq, num_kv_heads=hkv, head_dim=128,
+                         page_size=int(rng.choice([16, 32, 48, 128, 256])), seed=800 + seed, token_capacity=sum(ql) + 2,
+                         causal=bool(seed % 5 != 4))
+    rapi = binding.Rpa.for_meta(meta)
+    _, info = hz.full_parity(wl.materialize(meta, _dev(), canaries=bool(seed % 2)), rapi=rapi)
+    assert info["tile_kernel"] == 3
+    rapi.close()
