@@ -340,3 +340,41 @@ def test_plan_invariants_on_random_batches(seed):
     assert info["num_tokens"] == sum(q_lens)
     if threshold == 10 ** 6:
         assert info["num_tile_items"] == 0
+
+
+def test_pair_kernel_plans_cover_every_token_once_with_items_of_four_tiles():
+    """rpa_set_tile_pair(1) on a handle without a device: the plan's tile items hold up to four query tiles
+    (128 tokens at h_g = 4), never packed, one cache writer per (token, KV head), and the plan says which
+    kernel would run them; the default mode leaves plans of such handles on the two-tile kernel's items."""
+    build.build()
+    meta = wl.build_meta("pair_plan", [300, 64, 1, 129, 17], [811, 64, 500, 129, 17], seed=3, page_size=16, **wl.LLAMA3_8B)
+    r = binding.Rpa.for_meta(meta, device=-1)
+    r.rpa_plan(meta.cu_q_lens, meta.kv_lens)
+    info = r.rpa_plan_info()
+    assert info["tile_kernel"] == 1
+    default_tiles = info["num_tile_items"]
+    r.rpa_set_tile_pair(1)
+    r.rpa_plan(meta.cu_q_lens, meta.kv_lens)
+    info = r.rpa_plan_info()
+    rows, tiles, _ = r.rpa_plan_dump()
+    assert info["tile_kernel"] == 3 and 0 < info["num_tile_items"] < default_tiles
+    written = set()
+    for seq, head, tok0, n_tok, flags, n_seqs, _, _ in tiles:
+        assert 1 <= n_tok <= 128 and tok0 % 128 == 0 and not flags & 2  # kFlagPacked
+        assert tok0 + n_tok <= meta.q_lens[seq]
+        if flags & 1:  # kFlagWriteKv
+            for t in range(tok0, tok0 + n_tok):
+                assert (seq, head, t) not in written
+                written.add((seq, head, t))
+    for seq, head, tok0, n_tok, kv_begin, kv_end, partial, flags in rows:
+        if flags & 1:
+            for t in range(tok0, tok0 + n_tok):
+                assert (seq, head, t) not in written
+                written.add((seq, head, t))
+    assert len(written) == meta.num_kv_heads * meta.num_tokens
+    r.rpa_set_tile_pair(0)
+    r.rpa_plan(meta.cu_q_lens, meta.kv_lens)
+    assert r.rpa_plan_info()["num_tile_items"] == default_tiles
+    with pytest.raises(binding.RpaError):
+        r.rpa_set_tile_pair(7)
+    r.close()
