@@ -356,7 +356,7 @@ rpa_status_t rpa_set_tile_min_q(rpa_handle_t* h, int32_t tokens);
  * block (each stages half of it), with items of twice the tokens that follow one another without a
  * pause; it pays off where items are full.  mode 2 (the default): the pair kernel for pure long-prefill
  * batches (every sequence goes to the tile path and brings at least two full pair items of new
- * tokens), the two-tile kernel otherwise (mixed batches, small-q steps over long contexts, short
+ * tokens, and there are at least two pair items per SM), the two-tile kernel otherwise (mixed batches, small-q steps over long contexts, short
  * prompts).  mode 1: the pair kernel for every host-made plan with tile items (RPA_ERR_UNSUPPORTED
  * unless the cache is bf16 and d_k = 128).  mode 0: the two-tile kernel only.  Plans made on the device
  * and plans of handles without a device keep the two-tile kernel's items.  Invalidates the current

@@ -239,15 +239,17 @@ bool pair_kernel_wanted(const rpa_handle* h, const int32_t* cu_q_lens, const int
     if (h->plan_only && h->tile_pair_mode != 1) return false;  // (no device: plan what every device can run)
     if (h->tile_pair_mode == 1) return true;
     if (!cu_q_lens || !kv_lens) return false;
-    const int64_t long_q = 2 * tile2_kernel_tokens(h_g);
-    bool any = false;
+    const int64_t per_item = tile2_kernel_tokens(h_g), long_q = 2 * per_item;
+    int64_t items = 0;
     for (int32_t r = 0; r < num_seqs; ++r) {
         const int64_t q = (int64_t)cu_q_lens[r + 1] - cu_q_lens[r];
         if (q == 0) continue;
         if (!sequence_routed_to_tile(c, h->policy, q, kv_lens[r]) || q < long_q) return false;
-        any = true;
+        items += (int64_t)c.num_kv_heads * ((q + per_item - 1) / per_item);
     }
-    return any;
+    // ... and when there are enough items to keep every pair busy for a few rounds (one prompt of 2048
+    // tokens, 128 pair items on 74 pairs, ran 7 % slower than its 256 items on the two-tile kernel)
+    return items >= 2 * (int64_t)h->num_sms;
 }
 
 // Events recorded outside a capture cannot be waited for inside one (and the other way round): while

@@ -89,13 +89,23 @@ def test_pair_kernel_two_calls_on_one_handle_and_back_to_the_two_tile_kernel():
 
 def test_pair_kernel_is_chosen_for_long_prefill_only():
     # default mode: the pair kernel (items of 4 query tiles = 128 tokens at h_g = 4) when every sequence of the
-    # batch has at least 256 new tokens; a shorter sequence or a decode row keeps the batch on the two-tile kernel
-    for ql, kl, per_item in (([600, 300], [600, 1300], 128), ([600, 40], [600, 1300], 64), ([600, 300, 1], [600, 300, 900], 64)):
-        meta = wl.build_meta("pair_auto", ql, kl, num_q_heads=32, num_kv_heads=8, head_dim=128, page_size=16, seed=37)
+    # batch has at least 256 new tokens and there are at least two pair items per SM; a shorter sequence, a
+    # decode row or a batch too small to keep the pairs busy stays on the two-tile kernel
+    shape = dict(num_q_heads=32, num_kv_heads=8, head_dim=128, page_size=16)
+    for ql, kl, kernel in (([4800], [4800], 3), ([4800, 40], [4800, 1300], 1), ([4800, 1], [4800, 900], 1), ([600, 300], [600, 1300], 1)):
+        meta = wl.build_meta("pair_auto", ql, kl, seed=37, **shape)
         rapi = binding.Rpa.for_meta(meta)
-        _, info = hz.full_parity(wl.materialize(meta, _dev()), rapi=rapi)
+        rapi.rpa_plan(meta.cu_q_lens, meta.kv_lens)
+        info = rapi.rpa_plan_info()
+        assert info["tile_kernel"] == kernel
+        per_item = 128 if kernel == 3 else 64
         assert info["num_tile_items"] == 8 * sum(-(-q // per_item) for q in ql if q > 8)
         rapi.close()
+    meta = wl.build_meta("pair_auto", [4800], [4800], seed=38, **shape)
+    rapi = binding.Rpa.for_meta(meta)
+    _, info = hz.sampled_parity(wl.materialize(meta, _dev()), seqs=[0], rows_per_seq=160, whole_cache=True, rapi=rapi)
+    assert info["tile_kernel"] == 3
+    rapi.close()
 
 
 def test_device_planned_steps_keep_the_two_tile_kernel():
@@ -135,6 +145,7 @@ def test_pair_kernel_in_the_bounds_checked_build():
     tight = wl.build_meta("pair_dbg", [300, 260], [900, 260], num_q_heads=32, num_kv_heads=8, head_dim=128, page_size=16, seed=39,
                           pool_slack=1.0)
     rapi = binding.Rpa.for_meta(tight, library_path=debug_lib)
+    rapi.rpa_set_tile_pair(1)
     _, info = hz.full_parity(wl.materialize(tight, _dev(), canaries=True), rapi=rapi)
     assert info["tile_kernel"] == 3 and rapi.rpa_poll_status() == 0
     meta = dataclasses.replace(tight, num_pages=tight.num_pages + 8)  # the tensor holds 8 pages more than the handle knows of
@@ -158,7 +169,7 @@ def test_pair_kernel_in_the_bounds_checked_build():
 @pytest.mark.parametrize("seed", range(6))
 def test_pair_kernel_random_long_prefill_batches(seed):
     """Seeded random pure-prefill batches (ragged lengths from 256 tokens up, with and without cached context,
-    several head groupings and page sizes): whole-batch parity, automatic choice of the pair kernel."""
+    several head groupings and page sizes): whole-batch parity on the pair kernel."""
     rng = np.random.default_rng(4000 + seed)
     hq, hkv = [(32, 8), (16, 2), (8, 8), (32, 4), (16, 16), (64, 8)][seed % 6]
     tq4 = 4 * (128 // (hq // hkv))
@@ -168,7 +179,7 @@ def test_pair_kernel_random_long_prefill_batches(seed):
     meta = wl.build_meta(f"pair_rand{seed}", ql, kl, num_q_heads=hq, num_kv_heads=hkv, head_dim=128,
                          page_size=int(rng.choice([16, 32, 48, 128, 256])), seed=800 + seed, token_capacity=sum(ql) + 2,
                          causal=bool(seed % 5 != 4))
-    rapi = binding.Rpa.for_meta(meta)
+    rapi = _pair_api(meta)
     _, info = hz.full_parity(wl.materialize(meta, _dev(), canaries=bool(seed % 2)), rapi=rapi)
     assert info["tile_kernel"] == 3
     rapi.close()
