@@ -57,7 +57,6 @@ constexpr int kPairThreads = 384;  // 12 warps = 3 warpgroups per CTA
 constexpr int kPairWarps = 2 * (kPairThreads / 32);
 constexpr uint32_t kTmemCols = 512;
 constexpr float kRescaleThreshold = 8.f;  // log2 units
-constexpr int kBatchSpacing = 1040; // cycles between the product batches of the two tiles (see the MMA issuer)
 constexpr int kFetchAhead = 3;     // the next item is drawn when the running one has this many key blocks to go
 constexpr int D = 128;
 
@@ -374,17 +373,6 @@ rpa_tile2_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
         auto k_landed = [&](int f, uint32_t code) {  // fill f of the K ring, both halves
             return wait(BAR_KFULL + (f & 1), (f >> 1) & 1, code) && wait(BAR_KPEER + (f & 1), (f >> 1) & 1, code + 1);
         };
-        // The two tiles' softmax phases should not run at the same time: each runs at the special-
-        // function unit's full rate only when it has the unit to itself.  Nothing in the chain of
-        // dependencies sets the offset between the tiles, so the issuing warp does: a tile's batch of
-        // products (PV of this block, scores of the next) is not issued before `spacing` cycles have
-        // passed since the other tile's batch, which keeps the tiles about half a period apart.
-        const long long spacing = a.ablation >> 16 ? (long long)(a.ablation >> 16) * 16 : kBatchSpacing;
-        long long t_batch = clock64() - spacing;
-        auto keep_apart = [&]() {
-            while (clock64() - t_batch < spacing) {}
-            t_batch = clock64();
-        };
         int gb = 0;
         TileCtx it, nxt;
         int item, nxt_item = n_items;
@@ -400,8 +388,6 @@ rpa_tile2_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
                     tc_commit_pair(bar(BAR_SFULL + 0));
                 }
                 __syncwarp();
-                keep_apart();
-                keep_apart();
                 if (elect_one()) {
                     issue_qk(0, 1, 0, 0);
                     issue_qk(0, 1, 0, 1);
@@ -440,8 +426,7 @@ rpa_tile2_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
                     }
                     ok = wait(BAR_PREADY + 0, f & 1, 0x26);
                     if (!ok) break;
-                    keep_apart();
-                    tc_fence_after();
+                        tc_fence_after();
                     if (elect_one()) {
                         issue_pv(0, st, j == 0);
                         tc_commit_pair(bar(BAR_ODONE + 0));
@@ -461,8 +446,7 @@ rpa_tile2_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
                     }
                     ok = wait(BAR_PREADY + 1, f & 1, 0x27);
                     if (!ok) break;
-                    keep_apart();
-                    tc_fence_after();
+                        tc_fence_after();
                     if (elect_one()) {
                         issue_pv(1, st, j == 0);
                         tc_commit_pair(bar(BAR_ODONE + 1));
