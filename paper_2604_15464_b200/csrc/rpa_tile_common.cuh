@@ -153,13 +153,16 @@ __device__ __forceinline__ void tile_update_rounds(const KernelArgs& a, const Ti
     const int64_t tok_stride = (int64_t)a.h_kv * D;  // elements from one token's row to the next
     // writes a landed round out of its buffer; slot: this lane's token's cache slot in units of ROW
     // bytes (~0: none), read by the other lanes
+    // (a token's K row and V row sit side by side in the buffer, 2 * ROW bytes, as in the cache slot:
+    // lane t sends token t out with one bulk store - 32 instructions' worth of copy-engine work per
+    // round instead of 96 shuffles, loads and stores from a warp that is short of issue slots)
     auto write_out = [&](uint32_t buf, int nt, uint32_t slot) {
-#pragma unroll 4
-        for (int s = 0; s < STEPS; ++s) {
-            const int idx = s * 32 + lane, t = idx / CPT, piece = idx % CPT;
-            const uint32_t slot_t = __shfl_sync(0xffffffffu, slot, t);
-            if (t < nt && slot_t != ~0u) st_global_v4(cache + (int64_t)slot_t * ROW + piece * 16, ld_shared_v4(buf + idx * 16));
-        }
+        __syncwarp();                    // every lane's pieces have landed (each waited for its own copies)
+        sm100::fence_proxy_async_smem(); // ... and are visible to the copy engine
+        if (lane < nt && slot != ~0u) sm100::bulk_store(cache + (int64_t)slot * ROW, buf + lane * 2 * ROW, 2 * ROW);
+        sm100::bulk_commit();
+        sm100::bulk_wait_read();         // the buffer may be refilled
+        __syncwarp();
     };
     int r = 0, prev_nt = 0;
     uint32_t prev_slot = ~0u;
