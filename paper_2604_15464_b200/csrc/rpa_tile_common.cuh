@@ -118,14 +118,13 @@ __device__ __forceinline__ int packed_seq_of(const TileCtx& it, int tok) {
 // Fused cache update of an item ("Update U_kv" of Algorithm 1): the K and V rows of the item's own
 // tokens for its KV head go into their cache slots, a round of TPW tokens at a time.  The rows of a
 // round are fetched into shared memory with 16-byte asynchronous copies (one instruction moves 512
-// bytes for the warp and does not block it), then written out with 16-byte stores, 512 contiguous
-// bytes per token at d_k = 128 since K_h and V_h are neighbours in a slot.  (An earlier version gave
-// each lane a token and moved its rows with per-thread bulk copies: the copy engine takes such
-// copies one thread at a time, about 60 cycles each - 192 of them per 64 tokens, which is what an
-// item of a short prompt then cost.)  A lane computes the slot of "its" token of the round (token =
-// lane) and the others read it by shuffle; a lane stores exactly the bytes it fetched, so nothing
-// but its own wait orders the two.  BUFS: staging buffers of WARP_BYTES each; with two, the next
-// round's rows travel while this round's are written.
+// bytes for the warp and does not block it), a token's K row and V row side by side as in a cache
+// slot, and leave with one bulk store per token (lane t sends token t).  (An earlier version moved
+// the rows in both directions with per-thread bulk copies: the copy engine takes such copies one
+// thread at a time, about 60 cycles each - 192 of them per 64 tokens, which is what an item of a
+// short prompt then cost; 16-byte stores on the way out cost a shuffle, a shared-memory load and a
+// store per 512 bytes, more than the 32 bulk stores of a round.)  BUFS: staging buffers of
+// WARP_BYTES each; with two, the next round's rows travel while this round's are written.
 template <int D>
 struct TileUpdate {
     static constexpr int ROW_BYTES = D * 2;                       // one K or V row of one head
@@ -133,10 +132,6 @@ struct TileUpdate {
     static constexpr int WARP_BYTES = TPW * 2 * ROW_BYTES;
     static constexpr int STAGE_BYTES = 2 * WARP_BYTES;
 };
-
-__device__ __forceinline__ void st_global_v4(void* p, const uint4& v) {
-    asm volatile("st.global.v4.u32 [%0], {%1,%2,%3,%4};\n" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
-}
 
 // Rounds t_first, t_first + t_step, ... (token offsets inside the item) by one warp.  The warps of
 // the first warpgroup get an issue slot every few cycles only (the softmax warps own the schedulers),
@@ -152,10 +147,7 @@ __device__ __forceinline__ void tile_update_rounds(const KernelArgs& a, const Ti
     uint8_t* cache = reinterpret_cast<uint8_t*>(a.kv_cache);
     const int64_t tok_stride = (int64_t)a.h_kv * D;  // elements from one token's row to the next
     // writes a landed round out of its buffer; slot: this lane's token's cache slot in units of ROW
-    // bytes (~0: none), read by the other lanes
-    // (a token's K row and V row sit side by side in the buffer, 2 * ROW bytes, as in the cache slot:
-    // lane t sends token t out with one bulk store - 32 instructions' worth of copy-engine work per
-    // round instead of 96 shuffles, loads and stores from a warp that is short of issue slots)
+    // bytes (~0: none)
     auto write_out = [&](uint32_t buf, int nt, uint32_t slot) {
         __syncwarp();                    // every lane's pieces have landed (each waited for its own copies)
         sm100::fence_proxy_async_smem(); // ... and are visible to the copy engine

@@ -197,11 +197,13 @@ rpa_tile_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
             }
         };
         if (lane == 0) {
-            prefetch_tmap(&maps.q);
-            prefetch_tmap(&maps.out);
-            prefetch_tmap(&maps.cache);
-            prefetch_tmap(&maps.new_k);
-            prefetch_tmap(&maps.new_v);
+            if (iter == 0) {
+                prefetch_tmap(&maps.q);
+                prefetch_tmap(&maps.out);
+                prefetch_tmap(&maps.cache);
+                prefetch_tmap(&maps.new_k);
+                prefetch_tmap(&maps.new_v);
+            }
             if (q_prefetched_for != iter)  // the CTA's first item (later ones were loaded during their predecessor)
                 load_q(q_region, bar(BAR_Q + (iter & 1)), it.n_tok, h, cu + it.q_tok0);
         }
