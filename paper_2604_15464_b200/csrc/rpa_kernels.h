@@ -122,6 +122,8 @@ cudaError_t launch_quantise_q(const uint16_t* q, uint16_t* q_img, uint8_t* q_cod
 // several microseconds of host time, and a serving loop passes the same tensors step after step.  An
 // entry is reused when every tensor address and extent it was built from matches (a few entries, so
 // that alternating staging buffers all hit); null: encode afresh.
+constexpr int kTileMapBytes = 13 * 128;  // the CUtensorMap objects of one launch (128 bytes each)
+
 struct TileMapCache {
     static constexpr int kEntries = 4;
     struct Entry {
@@ -129,7 +131,7 @@ struct TileMapCache {
         const void *q = nullptr, *out = nullptr, *new_k = nullptr, *new_v = nullptr, *kv_cache = nullptr;
         int64_t token_rows = 0;
         int32_t h_q = 0, h_kv = 0, head_dim = 0, page_size = 0, num_pages = 0, kv_fp8 = 0, q_fp8 = 0, block_n = 0, q_tile_tokens = 0;
-        alignas(64) unsigned char maps[5 * 128];  // five CUtensorMap objects (128 bytes each)
+        alignas(64) unsigned char maps[kTileMapBytes];
     } entries[kEntries];
     int next = 0;
 };

@@ -11,12 +11,18 @@
 
 namespace rpa {
 
+constexpr int kUpdBoxes = 6;  // slot counts 1, 2, ..., 32 of one store of the fused cache update
+
 struct TileMaps {
     CUtensorMap q;      // (d, h_q, T)     box (64, G, query-tile tokens)
     CUtensorMap out;    // same geometry as q
     CUtensorMap new_k;  // (d, h_kv, T)    box (64, 1, key-block positions)
     CUtensorMap new_v;
     CUtensorMap cache;  // (d, 2h_kv, page_size, num_pages)  box (64, 1, page_box_rows(page_size, key-block positions), 1)
+    // fused cache update of a bf16 cache (whole rows, no swizzle): see tile_update_rounds_tma
+    CUtensorMap upd_k;  // (d, h_kv, T)    box (d, 1, TileUpdate<d>::TPW)
+    CUtensorMap upd_v;
+    CUtensorMap upd_cache[kUpdBoxes];  // (d, 2h_kv, page_size, num_pages)  box (d, 1, 1 << i, 1)
 };
 
 // Rows of one per-page TMA box of a context key block.  A block of block_n positions is fetched as
@@ -202,6 +208,64 @@ __device__ __forceinline__ void tile_update_rounds(const KernelArgs& a, const Ti
     }
 }
 
+// The same update with the copy engine doing all of it (bf16 cache): a round's K rows and V rows come
+// in as two boxes of TPW rows each (dense, K rows at `stage`, V rows behind them) and leave as a few
+// tiled stores.  The tokens of a round have consecutive positions, so they fall into runs that share
+// a page; a run of n slots goes out as one store per set bit of n (the largest first), K and V
+// apart - at a page size of 16, six to twelve stores a round where a store per token makes 32, and
+// two loads where 16-byte copies make 32 instructions.  `bar`: this warp's mbarrier (one arrival),
+// `parity` its running phase; `wait(bar, parity)` returns false when the kernel is being abandoned.
+template <int D, class Wait>
+__device__ __forceinline__ void tile_update_rounds_tma(const KernelArgs& a, const TileMaps& maps, const TileCtx& it, int t_first,
+                                                       int t_step, int lane, uint32_t stage, uint32_t bar, uint32_t& parity, Wait&& wait) {
+    using U = TileUpdate<D>;
+    constexpr int ROW = U::ROW_BYTES, TPW = U::TPW;
+    const int ps = a.page_size;
+    for (int t0 = t_first; t0 < it.n_tok; t0 += t_step) {
+        const int nt = min(TPW, it.n_tok - t0);
+        if (lane == 0) {
+            // (rows past the item's last token travel too and are not stored; past the tensor they read as zero)
+            sm100::mbar_arrive_expect_tx(bar, 2 * TPW * ROW);
+            sm100::tma_load_3d(stage, &maps.upd_k, 0, it.h, it.cu + it.q_tok0 + t0, bar);
+            sm100::tma_load_3d(stage + TPW * ROW, &maps.upd_v, 0, it.h, it.cu + it.q_tok0 + t0, bar);
+        }
+        const bool act = lane < nt;
+        const int tok = it.q_tok0 + t0 + lane;
+        int pos = it.c + tok;
+        const int32_t* pt_row = it.pt_row;
+        if (it.n_seqs > 1 && act) {  // packed item: the token's own sequence, page-table row and position
+            const int k = packed_seq_of(it, tok);
+            pos = tok - it.bounds[k];
+            pt_row += (int64_t)k * a.max_pages_per_seq;
+        }
+        const int page = act ? pt_row[pos / ps] : -1;
+        const bool valid = act && debug_write_page_ok(a, page);  // (always true for a token of the round outside the bounds-checked build)
+        // runs of tokens in one page: a run starts where the page changes (sequences share no page)
+        const int page_before = __shfl_up_sync(0xffffffffu, page, 1);
+        const bool valid_before = __shfl_up_sync(0xffffffffu, (int)valid, 1) != 0;
+        const uint32_t starts = __ballot_sync(0xffffffffu, !valid || lane == 0 || !valid_before || page != page_before);
+        int log_n = -1;  // this lane opens a store of 1 << log_n slots
+        if (valid) {
+            const int run0 = 31 - __clz(starts & (0xffffffffu >> (31 - lane)));
+            const uint32_t above = lane == 31 ? 0u : starts >> (lane + 1);
+            const int run_n = (above ? lane + __ffs(above) : 32) - run0;
+            const int rest = run_n - (lane - run0);  // slots of the run from this one on
+            const int hb = 31 - __clz(rest);
+            if (rest == (run_n & ((2 << hb) - 1))) log_n = hb;
+        }
+        const bool ok = wait(bar, parity);
+        parity ^= 1u;
+        if (ok && log_n >= 0) {
+            sm100::tma_store_4d(&maps.upd_cache[log_n], stage + lane * ROW, 0, 2 * it.h, pos % ps, page);
+            sm100::tma_store_4d(&maps.upd_cache[log_n], stage + (TPW + lane) * ROW, 0, 2 * it.h + 1, pos % ps, page);
+        }
+        sm100::bulk_commit();
+        sm100::bulk_wait_read();  // the buffer may be refilled
+        __syncwarp();
+        if (!ok) break;
+    }
+}
+
 // The update of one item shared by two warps (`w` = 0 or 1), each with its own staging buffer at
 // stage + w * WARP_BYTES: warp w takes every other round.
 template <int D>
@@ -291,9 +355,10 @@ inline EncodeTiledFn encode_fn() {
     return fn;
 }
 
-// tensor map (bf16 unless told otherwise) with 128-byte swizzle; dims/strides innermost first, strides in bytes for dims 1..
+// tensor map (bf16 and 128-byte swizzle unless told otherwise); dims/strides innermost first, strides in bytes for dims 1..
 inline bool make_map(CUtensorMap* m, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
-              const uint32_t* box, CUtensorMapDataType dtype = CU_TENSOR_MAP_DATA_TYPE_BFLOAT16) {
+              const uint32_t* box, CUtensorMapDataType dtype = CU_TENSOR_MAP_DATA_TYPE_BFLOAT16,
+              CUtensorMapSwizzle swizzle = CU_TENSOR_MAP_SWIZZLE_128B) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
     cuuint64_t gdim[5], gstr[5];
@@ -305,7 +370,7 @@ inline bool make_map(CUtensorMap* m, const void* base, int rank, const uint64_t*
         if (i > 0) gstr[i - 1] = strides_bytes[i - 1];
     }
     return fn(m, dtype, (cuuint32_t)rank, const_cast<void*>(base), gdim, gstr, bx, es,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -352,6 +417,19 @@ inline bool build_tile_maps(const KernelArgs& a, int64_t token_rows, int D, int 
         const uint64_t str[3] = {d * 2, d * 2 * 2 * a.h_kv, d * 2 * 2 * a.h_kv * a.page_size};
         const uint32_t box[4] = {64, 1, (uint32_t)page_box_rows(a.page_size, block_n), 1};
         if (!make_map(&maps->cache, a.kv_cache, 4, dims, str, box)) return false;
+        // the fused update's maps: whole rows as they lie in memory
+        const int tpw = 8192 / (2 * D) < 32 ? 8192 / (2 * D) : 32;  // TileUpdate<D>::TPW
+        const uint64_t ndims[3] = {d, (uint64_t)a.h_kv, (uint64_t)token_rows};
+        const uint64_t nstr[2] = {d * 2, d * 2 * a.h_kv};
+        const uint32_t nbox[3] = {(uint32_t)D, 1, (uint32_t)tpw};
+        if (!make_map(&maps->upd_k, a.new_k, 3, ndims, nstr, nbox, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, CU_TENSOR_MAP_SWIZZLE_NONE)) return false;
+        if (!make_map(&maps->upd_v, a.new_v, 3, ndims, nstr, nbox, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, CU_TENSOR_MAP_SWIZZLE_NONE)) return false;
+        for (int i = 0; i < kUpdBoxes; ++i) {
+            // (a store never leaves its page: a slot count above the page size or the round is never used)
+            const int n = (1 << i) <= a.page_size && (1 << i) <= tpw ? 1 << i : 1;
+            const uint32_t cbox[4] = {(uint32_t)D, 1, (uint32_t)n, 1};
+            if (!make_map(&maps->upd_cache[i], a.kv_cache, 4, dims, str, cbox, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, CU_TENSOR_MAP_SWIZZLE_NONE)) return false;
+        }
     }
     return true;
 }
@@ -360,7 +438,7 @@ inline bool build_tile_maps(const KernelArgs& a, int64_t token_rows, int D, int 
 // no entry was built from the same tensors.
 inline bool cached_tile_maps(TileMapCache* cache, const KernelArgs& a, int64_t token_rows, int D, int G, int q_tile_tokens,
                              int block_n, TileMaps* maps) {
-    static_assert(sizeof(TileMaps) == 5 * 128, "five tensor maps");
+    static_assert(sizeof(TileMaps) == kTileMapBytes, "thirteen tensor maps");
     if (!cache) return build_tile_maps(a, token_rows, D, G, q_tile_tokens, block_n, maps);
     const void* nk = a.q_fp8 ? (const void*)a.new_k_codes8 : a.kv_fp8 ? (const void*)a.new_k_codes : (const void*)a.new_k;
     const void* qp = a.q_fp8 ? (const void*)a.q_codes : (const void*)a.q;

@@ -132,20 +132,20 @@ rpa_tile_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
         mbar_init(bar(BAR_Q + 1), 1);
         fence_mbar_init();
     }
+    // Every barrier but BAR_Q starts afresh with each item, between the two CTA-wide barriers, at the
+    // hands of one thread, about 70 cycles a barrier.  Sharing the barriers out (one per lane of the
+    // producer warp, or a few per warp) lost arrivals: lane 0 of the four warps of the first
+    // warpgroup, with each barrier invalidated first, worked on short items and failed on long ones,
+    // every other split failed everywhere.  Invalidating each barrier before it is initialised again
+    // works with one thread too, but doubles the cost (2048 prompts of 64 tokens: 623 -> 683 us), so
+    // the barriers are initialised over their old state, as they always were; every one of them has
+    // completed its last phase and has no waiter by then.
     auto init_barriers = [&]() {
-        mbar_init(bar(BAR_NEXT), 1);
-        for (int s = 0; s < 2; ++s) {
-            mbar_init(bar(BAR_KFULL + s), 1);
-            mbar_init(bar(BAR_KEMPTY + s), 1);
-            mbar_init(bar(BAR_VFULL + s), 1);
-            mbar_init(bar(BAR_VEMPTY + s), 1);
-            mbar_init(bar(BAR_SFULL + s), 1);
-            mbar_init(bar(BAR_PREADY + s), 128);
-            mbar_init(bar(BAR_ODONE + s), 1);
-            mbar_init(bar(BAR_UPD + s), 1);
-            mbar_init(bar(BAR_EPI + s), 128);
-            mbar_init(bar(BAR_KCONV + s), 64);
-            mbar_init(bar(BAR_VCONV + s), 64);
+        for (int sl = BAR_KFULL; sl < BAR_COUNT; ++sl) {
+            const bool converters = sl >= BAR_KCONV && sl < BAR_VCONV + 2;
+            if (converters && !FP8) continue;  // (never used without an FP8 cache: still in their first phase)
+            const bool all_rows = sl == BAR_PREADY || sl == BAR_PREADY + 1 || sl == BAR_EPI || sl == BAR_EPI + 1;
+            mbar_init(bar(sl), all_rows ? 128 : converters ? 64 : 1);
         }
         fence_mbar_init();
     };
@@ -153,6 +153,7 @@ rpa_tile_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
       // first warpgroup: producer, MMA issuer, cache update; it needs few registers
       asm volatile("setmaxnreg.dec.sync.aligned.u32 56;\n");
       int q_prefetched_for = -1;  // producer: the iteration whose query tiles are already on their way
+      bool out_stores_pending = false;  // producer: output tiles of the previous item may still be leaving the V ring
       for (int iter = 0;; ++iter) {
       tc_fence_before();
       __syncthreads();  // everyone is done with the previous item
@@ -241,6 +242,11 @@ rpa_tile_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
             good = __all_sync(0xffffffffu, good);
             if (!good) return false;
             const uint32_t dst = (kv ? smem_base + C::OFF_V : k_region) + st * C::TILE_BYTES;
+            if (kv && out_stores_pending) {  // the previous item's output tiles were parked in the V ring
+                if (lane == 0) bulk_wait_read();
+                __syncwarp();
+                out_stores_pending = false;
+            }
             if (a.ablation & kAblateLoads) {
                 if (lane == 0) mbar_arrive(bar(full));
                 return true;
@@ -299,6 +305,26 @@ rpa_tile_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
                 if (lane == 0)
                     load_q(k_region, bar(BAR_Q + ((iter + 1) & 1)), nxt[RAW_NTOK], nxt[RAW_HEAD], nxt[RAW_CU] + nxt[RAW_TOK0]);
                 q_prefetched_for = iter + 1;
+            }
+        }
+        // The output tiles: the softmax groups park a full tile in the V ring (see the epilogue) and this
+        // warp hands it to the copy engine, so that no softmax thread waits for the store to read its
+        // tile out; the wait is taken before the next item's first V block instead.
+        if (ok && !(a.ablation & kAblateCompute) && !(it.n_tok <= TQ && n_blocks >= 2)) {
+            const int st_last = (n_blocks - 1) & 1;
+#pragma unroll
+            for (int x = 0; x < 2; ++x) {
+                if ((x + 1) * TQ > it.n_tok) break;
+                ok = mbar_wait(bar(BAR_EPI + x), 0, abort_flag, a.status, 0x36 + x);
+                if (!ok) break;
+                if (lane == 0) {
+                    const uint32_t o_buf = smem_base + C::OFF_V + (x == 0 ? st_last ^ 1 : st_last) * C::TILE_BYTES;
+#pragma unroll
+                    for (int b = 0; b < C::NBLK; ++b)
+                        tma_store_3d(&maps.out, o_buf + b * C::BLK_BYTES, b * 64, h * G, cu + it.q_tok0 + x * TQ);
+                    bulk_commit();
+                }
+                out_stores_pending = true;
             }
         }
       } else if (warp == 1) {
@@ -574,11 +600,16 @@ rpa_tile_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
                 }
             }
         } else if (!(a.ablation & kAblateUpdate) && (it.flags & kFlagWriteKv)) {
-            tile_update_cache<D>(a, it, warp - 2, lane, smem_base + C::OFF_UPD);
+            using U = TileUpdate<D>;
+            uint32_t parity = 0;  // (the barrier starts afresh with every item)
+            tile_update_rounds_tma<D>(a, maps, it, (warp - 2) * U::TPW, 2 * U::TPW, lane, smem_base + C::OFF_UPD + (warp - 2) * U::WARP_BYTES,
+                                      bar(BAR_UPD + warp - 2), parity,
+                                      [&](uint32_t b, uint32_t ph) { return mbar_wait(b, ph, abort_flag, a.status, 0x14); });
         }
         if (warp == 3 && !fetch_early) fetch_next();
       }
       }  // item loop of the first warpgroup
+      if (warp == 0 && lane == 0) bulk_wait_read();  // the last output tiles have left shared memory
     } else {
         // ================================ softmax warps ================================
         asm volatile("setmaxnreg.inc.sync.aligned.u32 224;\n");
@@ -767,11 +798,14 @@ rpa_tile_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
                     }
                 }
             } else if ((x + 1) * TQ <= it.n_tok) {
-                // A full tile goes out through shared memory: each thread parks its row in the
-                // tile's Q buffer (free since the last score product completed) in the swizzled
-                // layout of the tensor map, and one thread stores the tile with the copy engine.
-                // Row-per-thread stores to global would touch 32 lines per instruction.
-                const uint32_t q_buf = smem_base + q_off + x * C::TILE_BYTES;
+                // A full tile goes out through shared memory: each thread parks its row in the V
+                // ring, in the swizzled layout of the tensor map, and the producer warp stores the
+                // tile with the copy engine.  Row-per-thread stores to global would touch 32 lines per
+                // instruction.  Tile A, done first, takes the stage the last key block did not use
+                // (tile B's last PV product may still be reading that block's stage); tile B's own
+                // last product is the last reader of the other.
+                const int st_last = (n_blocks - 1) & 1;
+                const uint32_t q_buf = smem_base + C::OFF_V + (x == 0 ? st_last ^ 1 : st_last) * C::TILE_BYTES;
 #pragma unroll
                 for (int ch = 0; ch < D / 32; ++ch) {
                     uint32_t r32[32];
@@ -789,15 +823,6 @@ rpa_tile_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
                 }
                 fence_proxy_async_smem();
                 mbar_arrive(bar(BAR_EPI + x));
-                if (row == 0) {
-                    if (mbar_wait(bar(BAR_EPI + x), 0, abort_flag, a.status, 0x36 + x)) {
-#pragma unroll
-                        for (int b = 0; b < C::NBLK; ++b)
-                            tma_store_3d(&maps.out, q_buf + b * C::BLK_BYTES, b * 64, h * G, cu + it.q_tok0 + x * TQ);
-                        bulk_commit();
-                        bulk_wait_read();  // the Q buffer may be overwritten by the next item's load
-                    }
-                }
             } else {
                 uint16_t* dst = a.out + (((int64_t)cu + tok) * a.h_q + h * G + g) * D;
 #pragma unroll
