@@ -67,8 +67,11 @@ struct TileCfg {
 
 // barrier slots (8 bytes each) inside the barrier block
 // BAR_Q has one barrier per Q region and lives across items (a Q load for the next item may be in
-// flight while the others are re-initialised); BAR_NEXT: the next item's slot has been filled
-enum { BAR_Q = 0, BAR_KFULL = 2, BAR_KEMPTY = 4, BAR_VFULL = 6, BAR_VEMPTY = 8, BAR_SFULL = 10, BAR_PREADY = 12, BAR_ODONE = 14, BAR_UPD = 16, BAR_EPI = 18, BAR_KCONV = 20, BAR_VCONV = 22, BAR_NEXT = 24, BAR_COUNT = 25 };
+// flight while the others are re-initialised), and so does BAR_K0, on which an item's first key
+// block arrives (bf16 cache: it is fetched while the item before still runs); BAR_NEXT: the next
+// item's slot has been filled
+enum { BAR_Q = 0, BAR_K0 = 2, BAR_KFULL = 4, BAR_KEMPTY = 6, BAR_VFULL = 8, BAR_VEMPTY = 10, BAR_SFULL = 12, BAR_PREADY = 14, BAR_ODONE = 16, BAR_UPD = 18, BAR_EPI = 20, BAR_KCONV = 22, BAR_VCONV = 24, BAR_NEXT = 26, BAR_COUNT = 27 };
+static_assert(8 * BAR_COUNT + 24 <= 256, "barriers, abort flag, TMEM slot and progress fit below the item slots");
 
 
 // QF8 (FP8 cache with a per-tensor scale for Q as well, d_k = 128): the score product runs as
@@ -130,6 +133,8 @@ rpa_tile_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
     if (tid == 0) {
         mbar_init(bar(BAR_Q + 0), 1);
         mbar_init(bar(BAR_Q + 1), 1);
+        mbar_init(bar(BAR_K0 + 0), 1);
+        mbar_init(bar(BAR_K0 + 1), 1);
         fence_mbar_init();
     }
     // Every barrier but BAR_Q starts afresh with each item, between the two CTA-wide barriers, at the
@@ -153,6 +158,7 @@ rpa_tile_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
       // first warpgroup: producer, MMA issuer, cache update; it needs few registers
       asm volatile("setmaxnreg.dec.sync.aligned.u32 56;\n");
       int q_prefetched_for = -1;  // producer: the iteration whose query tiles are already on their way
+      int k0_prefetched_for = -1;  // producer: ... and whose first key block is
       bool out_stores_pending = false;  // producer: output tiles of the previous item may still be leaving the V ring
       for (int iter = 0;; ++iter) {
       tc_fence_before();
@@ -277,6 +283,33 @@ rpa_tile_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
             }
             return true;
         };
+        // First key block of an item (bf16 cache), into stage 0 of region `dst` on barrier `kbar`:
+        // of this item (the CTA's first) or, while this one still runs, of the next.
+        auto load_k0 = [&](const TileCtx& of, uint32_t dst, uint32_t kbar) {
+            if (a.ablation & kAblateLoads) {
+                if (lane == 0) mbar_arrive(kbar);
+                return;
+            }
+            if (of.n_ctx_blocks > 0) {
+                const int pos = lane * box_rows;
+                const bool sub_valid = lane < sub_blocks && pos < of.c;
+                int page = 0;
+                if (sub_valid) page = debug_read_page(a, of.pt_row[pos / ps]);
+                const int n_sub_valid = __popc(__ballot_sync(0xffffffffu, sub_valid));
+                if (lane == 0) mbar_arrive_expect_tx(kbar, (uint32_t)n_sub_valid * box_rows * D * 2);
+                __syncwarp();
+                if (sub_valid) {
+#pragma unroll
+                    for (int b = 0; b < C::NBLK; ++b)
+                        tma_load_4d(dst + b * C::BLK_BYTES + lane * box_rows * 128, &maps.cache, b * 64, 2 * of.h, pos % ps, page, kbar);
+                }
+            } else if (lane == 0) {
+                mbar_arrive_expect_tx(kbar, (uint32_t)C::TILE_BYTES);
+#pragma unroll
+                for (int b = 0; b < C::NBLK; ++b) tma_load_3d(dst + b * C::BLK_BYTES, &maps.new_k, b * 64, of.h, of.cu, kbar);
+            }
+        };
+        if (!FP8 && k0_prefetched_for != iter) load_k0(it, k_region, bar(BAR_K0 + (iter & 1)));
         // The keys run one block ahead of the values: K(j+1) goes out before V(j).  A V stage is held
         // much longer than a K stage (until the PV product of its block, i.e. through that block's whole
         // softmax), and with the loads in block order the wait for a free V stage also held back the
@@ -286,7 +319,13 @@ rpa_tile_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
             Src cur{0, 0, 0, false};
             if (t < n_blocks) {
                 cur = source_of(t);
-                ok = fill(t, 0, cur);
+                if (FP8 || t > 0) {
+                    ok = fill(t, 0, cur);
+                } else if (lane == 0) {
+                    // bf16 cache: block 0 is on its way already, on BAR_K0; stage 0's own barrier is
+                    // moved past its first phase, so that block 2k finds it in phase k as ever
+                    mbar_arrive(bar(BAR_KFULL + 0));
+                }
             }
             if (ok && t >= 1) ok = fill(t - 1, 1, prev);
             prev = cur;
@@ -305,6 +344,14 @@ rpa_tile_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
                 if (lane == 0)
                     load_q(k_region, bar(BAR_Q + ((iter + 1) & 1)), nxt[RAW_NTOK], nxt[RAW_HEAD], nxt[RAW_CU] + nxt[RAW_TOK0]);
                 q_prefetched_for = iter + 1;
+                if constexpr (!FP8) {
+                    // ... and its first key block, into this item's query region, which its last score
+                    // product has read (the output tiles are parked in the V ring): the next item's
+                    // first product then starts without the 1600 cycles a load takes to arrive
+                    const TileCtx nx = tile_ctx_from_raw(a, nxt, kBlockN);
+                    load_k0(nx, q_region, bar(BAR_K0 + ((iter + 1) & 1)));
+                    k0_prefetched_for = iter + 1;
+                }
             }
         }
         // The output tiles: the softmax groups park a full tile in the V ring (see the epilogue) and this
@@ -373,7 +420,11 @@ rpa_tile_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
         const bool two_tiles = it.n_tok > TQ;  // a short item (at most TQ tokens) runs tile A only
         const bool split = !two_tiles && n_blocks >= 2;  // ... with its key blocks dealt to both accumulators
         bool ok = mbar_wait(bar(BAR_Q + (iter & 1)), (iter >> 1) & 1, abort_flag, a.status, 0x20);
-        ok = ok && mbar_wait(k_ready(0), 0, abort_flag, a.status, 0x21);
+        if constexpr (FP8) {
+            ok = ok && mbar_wait(k_ready(0), 0, abort_flag, a.status, 0x21);
+        } else {
+            ok = ok && mbar_wait(bar(BAR_K0 + (iter & 1)), (iter >> 1) & 1, abort_flag, a.status, 0x21);
+        }
         if (split) {
             // Block j uses score buffer, accumulator and K/V stage j & 1, all with tile A's queries.
             // Order of issue: S_0, S_1, then per block O_x += P_j V_j followed by S_(j+2).
