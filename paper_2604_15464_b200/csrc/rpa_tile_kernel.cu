@@ -74,6 +74,56 @@ enum { BAR_Q = 0, BAR_K0 = 2, BAR_KFULL = 4, BAR_KEMPTY = 6, BAR_VFULL = 8, BAR_
 static_assert(8 * BAR_COUNT + 24 <= 256, "barriers, abort flag, TMEM slot and progress fit below the item slots");
 
 
+// Softmax of an item's only key block when at most half of it holds keys (a short prompt, a packed
+// item of short prompts): the scores of 64 positions come out of TMEM, the probabilities of the
+// other 64 are zero without an exponential being taken - with both tiles at once the exponentials
+// of 256 rows are what such an item waits for.  A function of its own, not inlined: the same
+// shortcut as a branch inside the kernel's softmax loop cost that loop 2 % on long prefill.
+// n_vis: visible positions of this thread's row from the block's start; n_before: positions at the
+// block's start that belong to earlier sequences of a packed item.  Returns the row's reference
+// maximum (log2 units, scaled) and sum.
+__device__ __noinline__ float2 softmax_half_block(uint32_t s_addr, int n_vis, int n_before, float scale_log2) {
+    constexpr int HALF = kBlockN / 2;
+    float s[HALF];
+#pragma unroll
+    for (int ch = 0; ch < HALF / 32; ++ch) {
+        uint32_t r32[32];
+        tmem_ld32(s_addr + ch * 32, r32);
+#pragma unroll
+        for (int i = 0; i < 32; ++i) s[ch * 32 + i] = __uint_as_float(r32[i]);
+    }
+    tc_wait_ld();
+#pragma unroll
+    for (int i = 0; i < HALF; ++i)
+        if (i >= n_vis || i < n_before) s[i] = -INFINITY;
+    float mxp[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) mxp[i] = fmaxf(s[i], s[i + 8]);
+#pragma unroll
+    for (int i = 16; i < HALF; i += 16)
+#pragma unroll
+        for (int k = 0; k < 8; ++k) mxp[k] = max3(mxp[k], s[i + k], s[i + k + 8]);
+    const float mx = fmaxf(max3(mxp[0], mxp[1], mxp[2]), max3(fmaxf(mxp[3], mxp[4]), max3(mxp[5], mxp[6], mxp[7]), -INFINITY));
+    const float m_ref = mx * scale_log2;
+    const float neg_m = m_ref == -INFINITY ? 0.f : -m_ref;
+    float lp[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+    uint32_t p32[32];
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+        float x0, x1;
+        fma2_bcast(x0, x1, s[2 * i], s[2 * i + 1], scale_log2, neg_m);
+        const float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
+        add2(lp[2 * (i & 3)], lp[2 * (i & 3) + 1], p0, p1);
+        p32[i] = pack_bf16x2(p0, p1);
+    }
+    tmem_st32(s_addr, p32);
+#pragma unroll
+    for (int i = 0; i < 32; ++i) p32[i] = 0u;
+    tmem_st32(s_addr + 32, p32);
+    tc_wait_st();
+    return make_float2(m_ref, ((lp[0] + lp[1]) + (lp[2] + lp[3])) + ((lp[4] + lp[5]) + (lp[6] + lp[7])));
+}
+
 // QF8 (FP8 cache with a per-tensor scale for Q as well, d_k = 128): the score product runs as
 // tcgen05.mma kind::f8f6f4 straight on code bytes - the query tile arrives as E4M3 codes (16 KB
 // instead of 32), a key block as the raw code rows of the cache (or of the scratch copy of the
@@ -704,6 +754,17 @@ rpa_tile_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
         bool ok = true;
         // tile B idles on a short item with a single key block
         const int my_blocks = split ? (n_blocks + 1 - x) >> 1 : (x == 1 && it.n_tok <= TQ) ? 0 : n_blocks;
+        if (n_blocks == 1 && n_new_visible <= kBlockN / 2 && my_blocks == 1 && !(a.ablation & kAblateCompute)) {
+            // the item's only block is at most half full (no context then: positions 0 .. n_new_visible - 1)
+            ok = mbar_wait(bar(BAR_SFULL + x), 0, abort_flag, a.status, 0x30 + x);
+            if (ok) {
+                tc_fence_after();
+                const float2 ml = softmax_half_block(s_addr, min(n_new_visible, lim + 1), packed ? first : 0, a.scale_log2);
+                m_ref = ml.x, l_sum = ml.y;
+                tc_fence_before();
+                mbar_arrive(bar(BAR_PREADY + x));
+            }
+        } else
         for (int jj = 0; jj < my_blocks; ++jj) {
             const int j = split ? 2 * jj + x : jj;  // key block; barrier phases count this group's own blocks
             ok = mbar_wait(bar(BAR_SFULL + x), jj & 1, abort_flag, a.status, 0x30 + x);
