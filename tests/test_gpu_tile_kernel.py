@@ -122,6 +122,29 @@ def test_packed_items_beside_context_and_decode_sequences():
     assert info["num_tile_items"] > 0 and info["num_row_items"] > 0
 
 
+HALF_BLOCK_CASES = [
+    # prompts without context whose only key block is at most half full (the softmax function of its own),
+    # many more items than CTAs: every CTA runs several, so the first key block of the next item, its query
+    # tiles and the output tiles of the one before are all in flight across item boundaries
+    # q_lens, h_q, h_kv, d, page_size, causal
+    ([64] * 40 + [33, 1, 64, 17] * 30, 32, 8, 128, 16, True),     # full and ragged tiles, one token, partial second tile
+    ([48, 64, 20] * 70, 32, 8, 128, 48, False),                     # no causal mask; pages that do not divide a block
+    ([64, 9, 64, 64, 31] * 20, 16, 16, 128, 16, True),              # h_g = 1: a 64-token prompt is half a query tile
+    ([64, 40] * 90, 16, 2, 64, 32, True),                           # d = 64, h_g = 8
+    # ... and beside items with a full block or several blocks (both softmax paths in one CTA's stream)
+    ([128, 64, 200, 30] * 40, 32, 8, 128, 16, True),
+]
+
+
+@pytest.mark.parametrize("case", HALF_BLOCK_CASES)
+def test_tile_kernel_items_of_a_single_half_full_block(case):
+    ql, hq, hkv, d, ps, causal = case
+    meta = wl.build_meta("half", ql, ql, num_q_heads=hq, num_kv_heads=hkv, head_dim=d, page_size=ps, seed=23,
+                         token_capacity=sum(ql) + 3, causal=causal)
+    _, info = hz.full_parity(wl.materialize(meta, _dev(), canaries=True), tile_min_q=1)
+    assert info["num_tile_items"] > 148 and info["num_row_items"] == 0 and info["tile_kernel"] == 1
+
+
 def test_tile_kernel_split_items_noncausal():
     meta = wl.build_meta("split-nc", [16, 30], [700, 129], num_q_heads=32, num_kv_heads=8, head_dim=128, page_size=16,
                          seed=17, causal=False)
