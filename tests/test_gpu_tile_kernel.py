@@ -145,6 +145,31 @@ def test_tile_kernel_items_of_a_single_half_full_block(case):
     assert info["num_tile_items"] > 148 and info["num_row_items"] == 0 and info["tile_kernel"] == 1
 
 
+@pytest.mark.parametrize("ql", [[64] * 3000, [128, 64, 300] * 400, [2048] * 6 + [40] * 500])
+def test_tile_kernel_repeated_launches_agree_bit_for_bit(ql):
+    """Persistent CTAs with many items each (loads, stores and barriers that live across item boundaries):
+    twelve launches of one plan must give the same bits every time, with nothing in the status word; the first
+    launch is checked against the oracle on sampled rows."""
+    meta = wl.build_meta("repeat", ql, ql, num_q_heads=32, num_kv_heads=8, head_dim=128, page_size=16, seed=27)
+    batch = wl.materialize(meta, _dev())
+    rapi = hz.binding.Rpa.for_meta(meta)
+    rapi.rpa_set_tile_pair(0)
+    _, info = hz.sampled_parity(batch, seqs=[0, len(ql) // 2, len(ql) - 1], rows_per_seq=48, whole_cache=True, rapi=rapi)
+    assert info["tile_kernel"] == 1 and info["num_tile_items"] > 4 * 148
+    first = None
+    for _ in range(12):
+        out = torch.zeros_like(batch.q)
+        rapi.rpa_forward(batch.q, batch.new_k, batch.new_v, batch.kv_cache, batch.page_table, batch.cu_q_lens, batch.kv_lens, out)
+        torch.cuda.synchronize()
+        assert rapi.rpa_poll_status() == 0
+        bits = wl.bf16_bits(out)
+        if first is None:
+            first = bits
+        else:
+            assert np.array_equal(first, bits)
+    rapi.close()
+
+
 def test_tile_kernel_split_items_noncausal():
     meta = wl.build_meta("split-nc", [16, 30], [700, 129], num_q_heads=32, num_kv_heads=8, head_dim=128, page_size=16,
                          seed=17, causal=False)
