@@ -27,6 +27,7 @@ struct rpa_handle {
     uint32_t ablation = 0;
     int tile_pair_mode = 2;  // tile items of host-made plans: 0 two-tile kernel, 1 CTA-pair kernel, 2 the pair kernel where every tile-routed sequence is long
     bool plan_pair = false;  // the current host-made plan's tile items are pair items
+    bool plan_short = false; // ... or all have at most two key blocks (see short_items_only)
     std::string last_error;
 
     // Device work lists, [row items | tile items | combine groups | kv_lens | cu_q_lens], in a ring of
@@ -252,6 +253,24 @@ bool pair_kernel_wanted(const rpa_handle* h, const int32_t* cu_q_lens, const int
     return items >= 2 * (int64_t)h->num_sms;
 }
 
+// The two-tile kernel has an instantiation for batches whose tile items all have one or two key blocks
+// (many short prompts without much context): there the per-item chain of latencies is everything, and
+// the cache update by the copy engine and the softmax function for a half-full block pay; on items
+// that stream many key blocks the same code costs 2-5 % (small-q steps over 4096 tokens of context on
+// 16-slot pages: 445 us with it, 426 without), so those keep the plain instantiation.
+bool short_items_only(const rpa_handle* h, const int32_t* cu_q_lens, const int32_t* kv_lens, int32_t num_seqs) {
+    const rpa_config_t& c = h->cfg;
+    if (c.kv_dtype != RPA_KV_BF16 || !cu_q_lens || !kv_lens) return false;
+    bool any = false;
+    for (int32_t r = 0; r < num_seqs; ++r) {
+        const int64_t q = (int64_t)cu_q_lens[r + 1] - cu_q_lens[r];
+        if (q == 0 || !sequence_routed_to_tile(c, h->policy, q, kv_lens[r])) continue;
+        if (kv_lens[r] > 2 * kQTile) return false;
+        any = true;
+    }
+    return any;
+}
+
 // Events recorded outside a capture cannot be waited for inside one (and the other way round): while
 // a stream is being captured into a graph, the capture's own order stands in for the handle's events.
 bool stream_is_capturing(cudaStream_t s) {
@@ -387,6 +406,7 @@ rpa_status_t rpa_plan(rpa_handle_t* h, const int32_t* cu_q_lens_host, const int3
     rpa_status_t st = build_plan(h->cfg, pol, cu_q_lens_host, kv_lens_host, num_seqs, h->plan);
     if (st != RPA_OK) return st;
     h->plan_pair = pair;
+    h->plan_short = !pair && short_items_only(h, cu_q_lens_host, kv_lens_host, num_seqs);
     h->plan.info.tile_kernel = h->plan.tiles.empty() ? 0
                                : pair ? 3
                                : tile1_kernel_supported(h->cfg.head_dim, h->cfg.num_q_heads / h->cfg.num_kv_heads) ? 2 : 1;
@@ -698,6 +718,7 @@ rpa_status_t rpa_forward(rpa_handle_t* h, const void* q, const void* new_k, cons
     a.num_row_items = (int32_t)h->plan.rows.size();
     a.num_tile_items = (int32_t)h->plan.tiles.size();
     a.num_tile_ctas = h->plan.tile_ctas;
+    a.short_items = h->plan_short ? 1 : 0;
     a.row_rows_max = h->plan.row_rows_max;
     a.num_groups = (int32_t)h->plan.groups.size();
     const bool fp8 = h->cfg.kv_dtype == RPA_KV_FP8_E4M3;

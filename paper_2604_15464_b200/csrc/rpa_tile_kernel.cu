@@ -129,7 +129,12 @@ __device__ __noinline__ float2 softmax_half_block(uint32_t s_addr, int n_vis, in
 // instead of 32), a key block as the raw code rows of the cache (or of the scratch copy of the
 // batch's own K codes), 32 elements of d_k per instruction at twice the bf16 rate - so no key is
 // expanded to bf16 any more; V keeps its bf16 expansion, P being bf16.
-template <int D, int G, bool FP8, bool QF8>
+//
+// SHORT: the instantiation for batches whose items all have one or two key blocks (bf16 cache): the
+// cache update goes through the copy engine and an item whose only block is at most half full takes
+// softmax_half_block.  Both are worth 10-20 % there and cost items that stream many key blocks
+// 2-5 % by their mere presence in the kernel, hence two instantiations.
+template <int D, int G, bool FP8, bool QF8, bool SHORT = false>
 __global__ void __launch_bounds__(kTileThreads, 1)
 rpa_tile_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
     static_assert(!QF8 || (FP8 && D == 128), "the FP8 score product is built for an FP8 cache and d_k = 128");
@@ -298,11 +303,6 @@ rpa_tile_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
             good = __all_sync(0xffffffffu, good);
             if (!good) return false;
             const uint32_t dst = (kv ? smem_base + C::OFF_V : k_region) + st * C::TILE_BYTES;
-            if (kv && out_stores_pending) {  // the previous item's output tiles were parked in the V ring
-                if (lane == 0) bulk_wait_read();
-                __syncwarp();
-                out_stores_pending = false;
-            }
             if (a.ablation & kAblateLoads) {
                 if (lane == 0) mbar_arrive(bar(full));
                 return true;
@@ -364,20 +364,28 @@ rpa_tile_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
         // much longer than a K stage (until the PV product of its block, i.e. through that block's whole
         // softmax), and with the loads in block order the wait for a free V stage also held back the
         // next block's keys, whose stage had long been free.
-        Src prev{0, 0, 0, false};
-        for (int t = 0; t <= n_blocks && ok; ++t) {
+        // (The loop is kept to what a block needs: this warp gets an issue slot every 60 cycles or so,
+        // and on 16-slot pages a block is 32 boxes.)
+        Src prev = source_of(0);
+        if constexpr (FP8) {
+            ok = fill(0, 0, prev);
+        } else if (lane == 0) {
+            // bf16 cache: block 0 is on its way already, on BAR_K0; stage 0's own barrier is moved past
+            // its first phase, so that block 2k finds it in phase k as ever
+            mbar_arrive(bar(BAR_KFULL + 0));
+        }
+        if (out_stores_pending) {  // the previous item's output tiles were parked in the V ring: before the first V block
+            if (lane == 0) bulk_wait_read();
+            __syncwarp();
+            out_stores_pending = false;
+        }
+        for (int t = 1; t <= n_blocks && ok; ++t) {
             Src cur{0, 0, 0, false};
             if (t < n_blocks) {
                 cur = source_of(t);
-                if (FP8 || t > 0) {
-                    ok = fill(t, 0, cur);
-                } else if (lane == 0) {
-                    // bf16 cache: block 0 is on its way already, on BAR_K0; stage 0's own barrier is
-                    // moved past its first phase, so that block 2k finds it in phase k as ever
-                    mbar_arrive(bar(BAR_KFULL + 0));
-                }
+                ok = fill(t, 0, cur);
             }
-            if (ok && t >= 1) ok = fill(t - 1, 1, prev);
+            if (ok) ok = fill(t - 1, 1, prev);
             prev = cur;
         }
         // the next item's query tiles, into this item's K ring once its last score product has read it
@@ -701,11 +709,15 @@ rpa_tile_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
                 }
             }
         } else if (!(a.ablation & kAblateUpdate) && (it.flags & kFlagWriteKv)) {
-            using U = TileUpdate<D>;
-            uint32_t parity = 0;  // (the barrier starts afresh with every item)
-            tile_update_rounds_tma<D>(a, maps, it, (warp - 2) * U::TPW, 2 * U::TPW, lane, smem_base + C::OFF_UPD + (warp - 2) * U::WARP_BYTES,
-                                      bar(BAR_UPD + warp - 2), parity,
-                                      [&](uint32_t b, uint32_t ph) { return mbar_wait(b, ph, abort_flag, a.status, 0x14); });
+            if constexpr (SHORT) {
+                using U = TileUpdate<D>;
+                uint32_t parity = 0;  // (the barrier starts afresh with every item)
+                tile_update_rounds_tma<D>(a, maps, it, (warp - 2) * U::TPW, 2 * U::TPW, lane, smem_base + C::OFF_UPD + (warp - 2) * U::WARP_BYTES,
+                                          bar(BAR_UPD + warp - 2), parity,
+                                          [&](uint32_t b, uint32_t ph) { return mbar_wait(b, ph, abort_flag, a.status, 0x14); });
+            } else {
+                tile_update_cache<D>(a, it, warp - 2, lane, smem_base + C::OFF_UPD);
+            }
         }
         if (warp == 3 && !fetch_early) fetch_next();
       }
@@ -754,7 +766,7 @@ rpa_tile_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
         bool ok = true;
         // tile B idles on a short item with a single key block
         const int my_blocks = split ? (n_blocks + 1 - x) >> 1 : (x == 1 && it.n_tok <= TQ) ? 0 : n_blocks;
-        if (n_blocks == 1 && n_new_visible <= kBlockN / 2 && my_blocks == 1 && !(a.ablation & kAblateCompute)) {
+        if (SHORT && n_blocks == 1 && n_new_visible <= kBlockN / 2 && my_blocks == 1 && !(a.ablation & kAblateCompute)) {
             // the item's only block is at most half full (no context then: positions 0 .. n_new_visible - 1)
             ok = mbar_wait(bar(BAR_SFULL + x), 0, abort_flag, a.status, 0x30 + x);
             if (ok) {
@@ -992,6 +1004,12 @@ cudaError_t launch_tile(const KernelArgs& a, int64_t token_rows, TileMapCache* c
             return cudaGetLastError();
         }
     }
+    if constexpr (!FP8) {
+        if (a.short_items && !a.dev_counts) {
+            rpa_tile_kernel<D, G, false, false, true><<<grid, kTileThreads, TileCfg<D>::SMEM, stream>>>(a, maps);
+            return cudaGetLastError();
+        }
+    }
     rpa_tile_kernel<D, G, FP8, false><<<grid, kTileThreads, TileCfg<D>::SMEM, stream>>>(a, maps);
     return cudaGetLastError();
 }
@@ -1000,6 +1018,10 @@ template <int D, int G, bool FP8>
 cudaError_t prepare_tile() {
     if constexpr (FP8 && D == 128) {
         cudaError_t e = cudaFuncSetAttribute(rpa_tile_kernel<D, G, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, TileCfg<D>::SMEM);
+        if (e != cudaSuccess) return e;
+    }
+    if constexpr (!FP8) {
+        cudaError_t e = cudaFuncSetAttribute(rpa_tile_kernel<D, G, false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, TileCfg<D>::SMEM);
         if (e != cudaSuccess) return e;
     }
     return cudaFuncSetAttribute(rpa_tile_kernel<D, G, FP8, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, TileCfg<D>::SMEM);
