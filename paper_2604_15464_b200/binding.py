@@ -52,7 +52,7 @@ class rpa_plan_info_t(ctypes.Structure):
                 ("gpu_launches", ctypes.c_int32), ("algorithmic_bytes", ctypes.c_int64),
                 ("algorithmic_flops", ctypes.c_int64), ("workspace_bytes", ctypes.c_int64),
                 ("row_bytes", ctypes.c_int64), ("tile_flops", ctypes.c_int64), ("tile_kernel", ctypes.c_int32),
-                ("reserved", ctypes.c_int32)]
+                ("tile_short_items", ctypes.c_int32)]
 
     def as_dict(self) -> dict:
         return {k: getattr(self, k) for k, _ in self._fields_}

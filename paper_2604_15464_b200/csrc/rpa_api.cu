@@ -220,7 +220,7 @@ void log_plan(const rpa_handle* h) {
             "%.3f GFLOP (row %.3f GB, tile %.3f GFLOP)\n",
             kCase[i.batch_case & 3], i.num_seqs, i.num_decode_seqs, i.num_prefill_seqs, i.num_tokens, i.num_row_items,
             h->plan.row_rows_max, i.kv_chunk_tokens, i.num_combine_groups, h->plan.num_partials,
-            i.tile_kernel == 3 ? "pair" : i.tile_kernel == 2 ? "single-tile" : "tile", i.num_tile_items,
+            i.tile_kernel == 3 ? "pair" : i.tile_kernel == 2 ? "single-tile" : i.tile_short_items ? "tile (short-item)" : "tile", i.num_tile_items,
             h->plan.tile_ctas > 0 ? h->plan.tile_ctas : (i.num_tile_items > 0 ? std::min(i.num_tile_items, h->num_sms) : 0),
             i.gpu_launches, i.algorithmic_bytes / 1e9, i.algorithmic_flops / 1e9, i.row_bytes / 1e9, i.tile_flops / 1e9);
 }
@@ -410,6 +410,8 @@ rpa_status_t rpa_plan(rpa_handle_t* h, const int32_t* cu_q_lens_host, const int3
     h->plan.info.tile_kernel = h->plan.tiles.empty() ? 0
                                : pair ? 3
                                : tile1_kernel_supported(h->cfg.head_dim, h->cfg.num_q_heads / h->cfg.num_kv_heads) ? 2 : 1;
+    h->plan_short = h->plan_short && h->plan.info.tile_kernel == 1;
+    h->plan.info.tile_short_items = h->plan_short ? 1 : 0;
     if (plan_log_enabled()) log_plan(h);
     if (!h->plan_only) {
         st = ensure_device(h);

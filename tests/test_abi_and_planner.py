@@ -342,6 +342,26 @@ def test_plan_invariants_on_random_batches(seed):
         assert info["num_tile_items"] == 0
 
 
+def test_short_item_instantiation_is_chosen_by_the_longest_tile_routed_sequence():
+    """The two-tile kernel's instantiation for short items: chosen when every sequence on the tile path has at
+    most 256 key positions (decode rows, which go to the row kernel, do not count), never for an FP8 cache."""
+    build.build()
+    shape = dict(seed=3, page_size=16, **wl.LLAMA3_8B)
+    for ql, kl, want in (([64] * 5, [64] * 5, 1), ([128, 200, 16], [128, 256, 16], 1), ([64, 1, 1], [64, 3000, 900], 1),
+                         ([64, 40], [64, 257], 0), ([300], [300], 0), ([1, 1], [500, 700], 0)):
+        meta = wl.build_meta("short_rule", ql, kl, **shape)
+        r = binding.Rpa.for_meta(meta, device=-1)
+        r.rpa_plan(meta.cu_q_lens, meta.kv_lens)
+        info = r.rpa_plan_info()
+        assert info["tile_short_items"] == want and (info["tile_kernel"] == 1 or not want)
+        r.close()
+    meta = wl.build_meta("short_rule_fp8", [64] * 5, [64] * 5, kv_fp8=True, k_scale=0.03, v_scale=0.03, **shape)
+    r = binding.Rpa.for_meta(meta, device=-1)
+    r.rpa_plan(meta.cu_q_lens, meta.kv_lens)
+    assert r.rpa_plan_info()["tile_short_items"] == 0
+    r.close()
+
+
 def test_pair_kernel_plans_cover_every_token_once_with_items_of_four_tiles():
     """rpa_set_tile_pair(1) on a handle without a device: the plan's tile items hold up to four query tiles
     (128 tokens at h_g = 4), never packed, one cache writer per (token, KV head), and the plan says which
