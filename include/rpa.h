@@ -123,9 +123,10 @@ typedef struct {
     int64_t tile_flops;         /* algorithmic FLOPs of the sequences served by the tile kernel      */
     int32_t tile_kernel;        /* which tensor-core kernel runs the tile items: 0 none, 1 two-tile,
                                    2 single-tile (d_k = 256), 3 CTA pair (see rpa_set_tile_pair)       */
-    int32_t tile_short_items;   /* 1: the two-tile kernel runs in its instantiation for short items (bf16
+    int32_t tile_short_items;   /* 1, 2: the two-tile kernel runs in its instantiation for short items (bf16
                                    cache, every sequence on the tile path has at most 256 key positions,
-                                   so every tile item has one or two key blocks); 0 otherwise          */
+                                   so every tile item has one or two key blocks; 2: at most 64, so every
+                                   item is one key block at most half full); 0 otherwise               */
 } rpa_plan_info_t;
 
 /*

@@ -27,7 +27,7 @@ struct rpa_handle {
     uint32_t ablation = 0;
     int tile_pair_mode = 2;  // tile items of host-made plans: 0 two-tile kernel, 1 CTA-pair kernel, 2 the pair kernel where every tile-routed sequence is long
     bool plan_pair = false;  // the current host-made plan's tile items are pair items
-    bool plan_short = false; // ... or all have at most two key blocks (see short_items_only)
+    int plan_short = 0;      // ... or all have at most two key blocks (1), at most half a block (2): see short_items_only
     std::string last_error;
 
     // Device work lists, [row items | tile items | combine groups | kv_lens | cu_q_lens], in a ring of
@@ -258,17 +258,19 @@ bool pair_kernel_wanted(const rpa_handle* h, const int32_t* cu_q_lens, const int
 // the cache update by the copy engine and the softmax function for a half-full block pay; on items
 // that stream many key blocks the same code costs 2-5 % (small-q steps over 4096 tokens of context on
 // 16-slot pages: 445 us with it, 426 without), so those keep the plain instantiation.
-bool short_items_only(const rpa_handle* h, const int32_t* cu_q_lens, const int32_t* kv_lens, int32_t num_seqs) {
+// Returns 0 (plain instantiation), 1 (short items) or 2 (short items that are all of one, at most
+// half-full key block: only then does the half-block softmax pay - in a batch that mixes such items
+// with full blocks, 1024 prompts of 128 tokens, it made the step 5-8 % slower).
+int short_items_only(const rpa_handle* h, const int32_t* cu_q_lens, const int32_t* kv_lens, int32_t num_seqs) {
     const rpa_config_t& c = h->cfg;
-    if (c.kv_dtype != RPA_KV_BF16 || !cu_q_lens || !kv_lens) return false;
-    bool any = false;
+    if (c.kv_dtype != RPA_KV_BF16 || !cu_q_lens || !kv_lens) return 0;
+    int32_t longest = 0;
     for (int32_t r = 0; r < num_seqs; ++r) {
         const int64_t q = (int64_t)cu_q_lens[r + 1] - cu_q_lens[r];
         if (q == 0 || !sequence_routed_to_tile(c, h->policy, q, kv_lens[r])) continue;
-        if (kv_lens[r] > 2 * kQTile) return false;
-        any = true;
+        longest = std::max(longest, kv_lens[r]);
     }
-    return any;
+    return longest == 0 || longest > 2 * kQTile ? 0 : longest <= kQTile / 2 ? 2 : 1;
 }
 
 // Events recorded outside a capture cannot be waited for inside one (and the other way round): while
@@ -406,12 +408,12 @@ rpa_status_t rpa_plan(rpa_handle_t* h, const int32_t* cu_q_lens_host, const int3
     rpa_status_t st = build_plan(h->cfg, pol, cu_q_lens_host, kv_lens_host, num_seqs, h->plan);
     if (st != RPA_OK) return st;
     h->plan_pair = pair;
-    h->plan_short = !pair && short_items_only(h, cu_q_lens_host, kv_lens_host, num_seqs);
+    h->plan_short = pair ? 0 : short_items_only(h, cu_q_lens_host, kv_lens_host, num_seqs);
     h->plan.info.tile_kernel = h->plan.tiles.empty() ? 0
                                : pair ? 3
                                : tile1_kernel_supported(h->cfg.head_dim, h->cfg.num_q_heads / h->cfg.num_kv_heads) ? 2 : 1;
-    h->plan_short = h->plan_short && h->plan.info.tile_kernel == 1;
-    h->plan.info.tile_short_items = h->plan_short ? 1 : 0;
+    if (h->plan.info.tile_kernel != 1) h->plan_short = 0;
+    h->plan.info.tile_short_items = h->plan_short;
     if (plan_log_enabled()) log_plan(h);
     if (!h->plan_only) {
         st = ensure_device(h);
@@ -720,7 +722,7 @@ rpa_status_t rpa_forward(rpa_handle_t* h, const void* q, const void* new_k, cons
     a.num_row_items = (int32_t)h->plan.rows.size();
     a.num_tile_items = (int32_t)h->plan.tiles.size();
     a.num_tile_ctas = h->plan.tile_ctas;
-    a.short_items = h->plan_short ? 1 : 0;
+    a.short_items = h->plan_short;
     a.row_rows_max = h->plan.row_rows_max;
     a.num_groups = (int32_t)h->plan.groups.size();
     const bool fp8 = h->cfg.kv_dtype == RPA_KV_FP8_E4M3;

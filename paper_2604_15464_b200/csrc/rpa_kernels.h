@@ -56,7 +56,7 @@ struct KernelArgs {
     int32_t kv_fp8;    // cache elements are FP8 E4M3 bytes
     int32_t validated; // a validation kernel ran before this launch: leave at once if it flagged the inputs
     uint32_t ablation;
-    int32_t short_items;  // two-tile kernel: every tile item has at most two key blocks (chooses the instantiation built for such items)
+    int32_t short_items;  // two-tile kernel: 1 every tile item has at most two key blocks (chooses the instantiation built for such items), 2 each is one block at most half full
     // Lists planned on the device: the counts live in device memory (written by the plan kernel of the
     // same step) and take the place of num_row_items, num_tile_items, num_groups and num_tile_ctas.
     const int32_t* dev_counts;  // null: the counts above hold

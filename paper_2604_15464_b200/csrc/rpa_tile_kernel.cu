@@ -766,7 +766,7 @@ rpa_tile_kernel(const KernelArgs a, const __grid_constant__ TileMaps maps) {
         bool ok = true;
         // tile B idles on a short item with a single key block
         const int my_blocks = split ? (n_blocks + 1 - x) >> 1 : (x == 1 && it.n_tok <= TQ) ? 0 : n_blocks;
-        if (SHORT && n_blocks == 1 && n_new_visible <= kBlockN / 2 && my_blocks == 1 && !(a.ablation & kAblateCompute)) {
+        if (SHORT && a.short_items == 2 && n_blocks == 1 && n_new_visible <= kBlockN / 2 && my_blocks == 1 && !(a.ablation & kAblateCompute)) {
             // the item's only block is at most half full (no context then: positions 0 .. n_new_visible - 1)
             ok = mbar_wait(bar(BAR_SFULL + x), 0, abort_flag, a.status, 0x30 + x);
             if (ok) {

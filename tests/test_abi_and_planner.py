@@ -344,10 +344,11 @@ def test_plan_invariants_on_random_batches(seed):
 
 def test_short_item_instantiation_is_chosen_by_the_longest_tile_routed_sequence():
     """The two-tile kernel's instantiation for short items: chosen when every sequence on the tile path has at
-    most 256 key positions (decode rows, which go to the row kernel, do not count), never for an FP8 cache."""
+    most 256 key positions (2: at most 64; decode rows, which go to the row kernel, do not count), never for an FP8
+    cache."""
     build.build()
     shape = dict(seed=3, page_size=16, **wl.LLAMA3_8B)
-    for ql, kl, want in (([64] * 5, [64] * 5, 1), ([128, 200, 16], [128, 256, 16], 1), ([64, 1, 1], [64, 3000, 900], 1),
+    for ql, kl, want in (([64] * 5, [64] * 5, 2), ([128, 200, 16], [128, 256, 16], 1), ([64, 1, 1], [64, 3000, 900], 2), ([65], [65], 1),
                          ([64, 40], [64, 257], 0), ([300], [300], 0), ([1, 1], [500, 700], 0)):
         meta = wl.build_meta("short_rule", ql, kl, **shape)
         r = binding.Rpa.for_meta(meta, device=-1)

@@ -143,7 +143,7 @@ def test_tile_kernel_items_of_a_single_half_full_block(case):
                          token_capacity=sum(ql) + 3, causal=causal)
     _, info = hz.full_parity(wl.materialize(meta, _dev(), canaries=True), tile_min_q=1)
     assert info["num_tile_items"] > 148 and info["num_row_items"] == 0 and info["tile_kernel"] == 1
-    assert info["tile_short_items"] == (1 if max(ql) <= 256 else 0)
+    assert info["tile_short_items"] == (2 if max(ql) <= 64 else 1 if max(ql) <= 256 else 0)
 
 
 @pytest.mark.parametrize("ql", [[64] * 3000, [128, 64, 300] * 400, [2048] * 6 + [40] * 500])
